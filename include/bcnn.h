@@ -1,0 +1,141 @@
+/*
+ * bcnn.h - C ABI of the binary (+-1 x +-1) convolution library for NVIDIA B200 (sm_100a).
+ *
+ * The operator is the CNN-style 2D convolution of the paper (Section 1: 3D input
+ * tensor, 4D weight tensor, 3D output tensor, lowered to a matrix-matrix product)
+ * with both operands binarized (Section 4.2.1: every feature is +1 or -1 and every
+ * weight is +1 or -1; Section 5.2 / Figure 5: forward weights are the sign of the
+ * real weights).  For +-1 vectors the inner product over K elements equals
+ * K - 2*popcount(a XOR w) on their sign bits; the library computes exactly that
+ * integer.
+ *
+ * Conventions shared by every call
+ *   - Sign-bit encoding: bit 1 = +1, bit 0 = -1.
+ *   - Packed activations are NHWC; the C channels of one pixel occupy C/8 consecutive
+ *     bytes, channel c in byte c/8, bit c%8 (LSB first).  Read as little-endian 32- or
+ *     64-bit words this is the same memory.  C must be a multiple of 32.
+ *   - Packed weights are [C_out][kh][kw][C_in] with C_in packed the same way, i.e.
+ *     N = C_out rows of K = kh*kw*C_in bits.  A GEMM "B" operand is likewise N rows
+ *     of K bits (the K x N matrix stored column by column).
+ *   - Out-of-image taps of a convolution read the value -1 (a +-1 tensor has no
+ *     zero); BCNN_PAD_VALUE documents it.  K in "K - 2*popcount" is always the full
+ *     kh*kw*C_in.
+ *   - Output extent: OH = floor((H + 2*pad - kh)/stride) + 1, same for OW.
+ *   - All data pointers are DEVICE pointers owned by the caller, 16-byte aligned.
+ *     The library never allocates, frees or synchronises: every call only enqueues
+ *     kernels on `stream` (a cudaStream_t passed as void*, NULL = default stream)
+ *     and returns.  Buffers may be reused as soon as the stream has passed the call.
+ *   - Every call validates its arguments first and launches nothing on error.
+ *     Return value: BCNN_OK or a negative bcnn_status.
+ */
+#ifndef BCNN_H
+#define BCNN_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define BCNN_PAD_VALUE (-1)
+
+typedef enum bcnn_status {
+    BCNN_OK = 0,
+    BCNN_ERR_INVALID_ARG = -1, /* null pointer, non-positive size, empty output */
+    BCNN_ERR_UNSUPPORTED = -2, /* channel count not a multiple of 32, size limits */
+    BCNN_ERR_ALIGNMENT = -3,   /* a data pointer is not 16-byte aligned */
+    BCNN_ERR_CUDA = -4         /* the CUDA runtime refused a launch */
+} bcnn_status;
+
+/* Engines of the inner product; BCNN_ENGINE_AUTO picks per shape. */
+typedef enum bcnn_engine {
+    BCNN_ENGINE_AUTO = 0,
+    BCNN_ENGINE_LOP3 = 1,   /* CUDA cores: XOR + popcount                              */
+    BCNN_ENGINE_MMA_B1 = 2, /* warp-level mma.sync m16n8k256 .b1 AND + popcount         */
+    BCNN_ENGINE_TC_I8 = 3   /* sign bits expanded to int8 in shared memory, tcgen05 i8  */
+} bcnn_engine;
+
+/*
+ * Binarize and pack (Section 4.2.1: learnable bias, then sign; Section 4.2.2: channel
+ * replication by an integer factor R is bookkeeping, not a copy).
+ *   out bit[b][h][w][c] = (x[b][h][w][c mod C_in] + bias[c] >= 0),  c in [0, R*C_in)
+ * The add is an fp32 add, the compare is >= 0 (so -0.0 -> +1, NaN -> -1).
+ *   x        device, fp32 NHWC [B][H][W][C_in]
+ *   bias     device, fp32 [R*C_in], or NULL for no bias
+ *   out_bits device, B*H*W*(R*C_in)/8 bytes, layout above; R*C_in % 32 == 0
+ * With B = C_out, H = kh, W = kw the same call packs real weights into the weight
+ * layout (Section 5.2).
+ */
+int bcnn_pack(const float *x, const float *bias, void *out_bits,
+              int B, int H, int W, int C_in, int R, void *stream);
+
+/*
+ * Binary matrix product (Section 1 lowering):
+ *   C[m][n] = sum_k a[m][k]*w[n][k] = K - 2*popcount(A_m XOR W_n),  a, w in {-1,+1}
+ *   A_bits device, M rows of K bits;  W_bits device, N rows of K bits;  K % 32 == 0
+ *   C      device, int32 [M][N] row-major
+ */
+int bcnn_gemm_b1(const void *A_bits, const void *W_bits, int32_t *C,
+                 int64_t M, int N, int K, void *stream);
+
+/*
+ * The same product followed by a per-column integer threshold that emits packed sign
+ * bits (Section 4.2.1: batch norm scale/bias and the next module's bias + sign, folded
+ * into one integer comparison):
+ *   out bit[m][n] = (C[m][n] >= thr[n])
+ *   thr      device, int32 [N];  out_bits device, M rows of N bits;  N % 32 == 0
+ * A batch norm with negative scale is folded by the caller: flip that channel's weight
+ * bits and negate its threshold.
+ */
+int bcnn_gemm_b1_fused(const void *A_bits, const void *W_bits, const int32_t *thr,
+                       void *out_bits, int64_t M, int N, int K, void *stream);
+
+/*
+ * Binary convolution as an implicit GEMM (the patch matrix is never materialised):
+ *   y[b][oh][ow][co] = sum_{r,t,ci} xpad[b][oh*stride-pad+r][ow*stride-pad+t][ci] * w[co][r][t][ci]
+ * with xpad = x inside the image and -1 outside.
+ *   x_bits device, packed NHWC [B][H][W][C_in];  w_bits device, packed [C_out][kh][kw][C_in]
+ *   y      device, int32 NHWC [B][OH][OW][C_out]
+ *   C_in % 32 == 0; kh, kw >= 1; stride >= 1; pad >= 0; OH, OW >= 1; B*OH*OW < 2^31
+ */
+int bcnn_conv2d_b1(const void *x_bits, const void *w_bits, int32_t *y,
+                   int B, int H, int W, int C_in, int C_out,
+                   int kh, int kw, int stride, int pad, void *stream);
+
+/*
+ * Convolution with the fused threshold / re-pack epilogue: the output is the next
+ * layer's packed input, y bit[b][oh][ow][co] = (acc >= thr[co]).
+ *   thr device int32 [C_out];  y_bits device, packed NHWC [B][OH][OW][C_out];  C_out % 32 == 0
+ */
+int bcnn_conv2d_b1_fused(const void *x_bits, const void *w_bits, const int32_t *thr,
+                         void *y_bits, int B, int H, int W, int C_in, int C_out,
+                         int kh, int kw, int stride, int pad, void *stream);
+
+/*
+ * The same four products with the inner-product engine chosen by the caller (used to
+ * compare engines; BCNN_ENGINE_AUTO behaves like the calls above).  thr == NULL selects
+ * the int32 output (`out` is int32), otherwise the packed output.  Returns
+ * BCNN_ERR_UNSUPPORTED when the engine cannot run the shape.
+ */
+int bcnn_conv2d_b1_engine(int engine, const void *x_bits, const void *w_bits, const int32_t *thr,
+                          void *out, int B, int H, int W, int C_in, int C_out,
+                          int kh, int kw, int stride, int pad, void *stream);
+int bcnn_gemm_b1_engine(int engine, const void *A_bits, const void *W_bits, const int32_t *thr,
+                        void *out, int64_t M, int N, int K, void *stream);
+
+/*
+ * Device-side error word.  Kernels that wait on hardware barriers give up after a
+ * bounded number of polls and record a non-zero code here instead of hanging.
+ * Reads the word of the current device (synchronises that device) and clears it.
+ * Returns the code (0 = no error) or a negative bcnn_status.
+ */
+int bcnn_device_error(void);
+
+const char *bcnn_status_string(int status);
+int bcnn_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* BCNN_H */

@@ -1,0 +1,122 @@
+"""Thin ctypes binding of the C ABI in include/bcnn.h.
+
+Argument marshalling only: every step of the path runs in the CUDA kernels.  Tensors
+are torch CUDA tensors used purely as device buffers; the functions take their
+``data_ptr()`` and the current torch stream.  There is no CPU fallback: if the shared
+library is missing or does not load, importing the symbols raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+
+import torch
+
+_PKG = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_PKG, "libbcnn.so")
+
+ENGINE_AUTO, ENGINE_LOP3, ENGINE_MMA_B1, ENGINE_TC_I8 = 0, 1, 2, 3
+ENGINES = {"auto": ENGINE_AUTO, "lop3": ENGINE_LOP3, "mma_b1": ENGINE_MMA_B1, "tc_i8": ENGINE_TC_I8}
+
+EXPORTS = (
+    "bcnn_pack", "bcnn_gemm_b1", "bcnn_gemm_b1_fused", "bcnn_conv2d_b1", "bcnn_conv2d_b1_fused",
+    "bcnn_conv2d_b1_engine", "bcnn_gemm_b1_engine", "bcnn_device_error", "bcnn_status_string",
+    "bcnn_version",
+)
+
+_lib = None
+
+
+class BcnnError(RuntimeError):
+    def __init__(self, status: int, what: str):
+        self.status = status
+        super().__init__(f"{what}: {status_string(status)} ({status})")
+
+
+def load() -> ctypes.CDLL:
+    """Load libbcnn.so (built in-tree by ``build.py``); raises if it is absent."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise ImportError(f"{LIB_PATH} not built: run python -m paper_2010_00704_b200.build")
+        lib = ctypes.CDLL(LIB_PATH)
+        vp, i32, i64 = ctypes.c_void_p, ctypes.c_int, ctypes.c_int64
+        lib.bcnn_pack.argtypes = [vp, vp, vp, i32, i32, i32, i32, i32, vp]
+        lib.bcnn_gemm_b1.argtypes = [vp, vp, vp, i64, i32, i32, vp]
+        lib.bcnn_gemm_b1_fused.argtypes = [vp, vp, vp, vp, i64, i32, i32, vp]
+        lib.bcnn_conv2d_b1.argtypes = [vp, vp, vp] + [i32] * 9 + [vp]
+        lib.bcnn_conv2d_b1_fused.argtypes = [vp, vp, vp, vp] + [i32] * 9 + [vp]
+        lib.bcnn_conv2d_b1_engine.argtypes = [i32, vp, vp, vp, vp] + [i32] * 9 + [vp]
+        lib.bcnn_gemm_b1_engine.argtypes = [i32, vp, vp, vp, vp, i64, i32, i32, vp]
+        lib.bcnn_device_error.argtypes = []
+        lib.bcnn_status_string.argtypes = [i32]
+        lib.bcnn_status_string.restype = ctypes.c_char_p
+        for name in EXPORTS:
+            if name != "bcnn_status_string":
+                getattr(lib, name).restype = i32
+        _lib = lib
+    return _lib
+
+
+def status_string(status: int) -> str:
+    return load().bcnn_status_string(int(status)).decode()
+
+
+def version() -> int:
+    return load().bcnn_version()
+
+
+def _stream() -> int:
+    return torch.cuda.current_stream().cuda_stream
+
+
+def _p(t) -> int | None:
+    return None if t is None else t.data_ptr()
+
+
+def _check(status: int, what: str):
+    if status != 0:
+        raise BcnnError(status, what)
+
+
+def out_hw(H, W, kh, kw, stride, pad):
+    return (H + 2 * pad - kh) // stride + 1, (W + 2 * pad - kw) // stride + 1
+
+
+def bcnn_pack(x: torch.Tensor, bias, out_bits: torch.Tensor, B, H, W, C_in, R=1):
+    """x fp32 NHWC device tensor -> packed sign bits written into ``out_bits``."""
+    _check(load().bcnn_pack(_p(x), _p(bias), _p(out_bits), B, H, W, C_in, R, _stream()), "bcnn_pack")
+    return out_bits
+
+
+def bcnn_gemm_b1(A_bits, W_bits, C, M, N, K, engine=ENGINE_AUTO):
+    _check(load().bcnn_gemm_b1_engine(engine, _p(A_bits), _p(W_bits), None, _p(C), M, N, K, _stream()),
+           "bcnn_gemm_b1")
+    return C
+
+
+def bcnn_gemm_b1_fused(A_bits, W_bits, thr, out_bits, M, N, K, engine=ENGINE_AUTO):
+    if thr is None:
+        raise BcnnError(-1, "bcnn_gemm_b1_fused")
+    _check(load().bcnn_gemm_b1_engine(engine, _p(A_bits), _p(W_bits), _p(thr), _p(out_bits), M, N, K, _stream()),
+           "bcnn_gemm_b1_fused")
+    return out_bits
+
+
+def bcnn_conv2d_b1(x_bits, w_bits, y, B, H, W, C_in, C_out, kh, kw, stride, pad, engine=ENGINE_AUTO):
+    _check(load().bcnn_conv2d_b1_engine(engine, _p(x_bits), _p(w_bits), None, _p(y), B, H, W, C_in, C_out,
+                                        kh, kw, stride, pad, _stream()), "bcnn_conv2d_b1")
+    return y
+
+
+def bcnn_conv2d_b1_fused(x_bits, w_bits, thr, y_bits, B, H, W, C_in, C_out, kh, kw, stride, pad,
+                         engine=ENGINE_AUTO):
+    if thr is None:
+        raise BcnnError(-1, "bcnn_conv2d_b1_fused")
+    _check(load().bcnn_conv2d_b1_engine(engine, _p(x_bits), _p(w_bits), _p(thr), _p(y_bits), B, H, W, C_in,
+                                        C_out, kh, kw, stride, pad, _stream()), "bcnn_conv2d_b1_fused")
+    return y_bits
+
+
+def bcnn_device_error() -> int:
+    return load().bcnn_device_error()

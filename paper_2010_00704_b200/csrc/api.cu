@@ -1,0 +1,163 @@
+// C ABI: argument validation, problem set-up and engine dispatch.  No allocation,
+// no synchronisation: every entry point only enqueues kernels on the caller's stream.
+#include "bcnn_common.cuh"
+
+namespace bcnn {
+
+__device__ int g_device_error = 0;
+
+namespace {
+
+inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+int make_conv_problem(ConvProblem &p, const void *x, const void *w, const int32_t *thr, void *out,
+                      int B, int H, int W, int C_in, int C_out, int kh, int kw, int stride, int pad,
+                      bool fused)
+{
+    if (!x || !w || !out || (fused && !thr)) return BCNN_ERR_INVALID_ARG;
+    if (B <= 0 || H <= 0 || W <= 0 || C_in <= 0 || C_out <= 0 || kh <= 0 || kw <= 0 || stride <= 0 || pad < 0)
+        return BCNN_ERR_INVALID_ARG;
+    if (H + 2 * (long)pad < kh || W + 2 * (long)pad < kw) return BCNN_ERR_INVALID_ARG;
+    if (C_in % 32 != 0) return BCNN_ERR_UNSUPPORTED;
+    if (fused && C_out % 32 != 0) return BCNN_ERR_UNSUPPORTED;
+    if (!aligned16(x) || !aligned16(w) || !aligned16(out) || (thr && !aligned16(thr))) return BCNN_ERR_ALIGNMENT;
+    const long OH = (H + 2L * pad - kh) / stride + 1;
+    const long OW = (W + 2L * pad - kw) / stride + 1;
+    const long M = (long)B * OH * OW;
+    const long K = (long)kh * kw * C_in;
+    if (M >= (1L << 31) || K >= (1L << 30)) return BCNN_ERR_UNSUPPORTED;
+    if ((long)B * H * W * (C_in / 32) >= (1L << 40)) return BCNN_ERR_UNSUPPORTED;
+    p.x = static_cast<const uint32_t *>(x);
+    p.w = static_cast<const uint32_t *>(w);
+    p.thr = fused ? thr : nullptr;
+    p.out = out;
+    p.B = B; p.H = H; p.W = W; p.C_in = C_in; p.C_out = C_out;
+    p.kh = kh; p.kw = kw; p.stride = stride; p.pad = pad;
+    p.OH = (int)OH; p.OW = (int)OW;
+    p.cw = C_in / 32;
+    p.K = (int)K;
+    p.kwords = (int)(K / 32);
+    p.M = (int)M;
+    return BCNN_OK;
+}
+
+int dispatch(int engine, const ConvProblem &p, cudaStream_t stream)
+{
+    switch (engine) {
+    case BCNN_ENGINE_AUTO:
+        if (conv_mma_b1_supports(p)) return launch_conv_mma_b1(p, stream);
+        return launch_conv_lop3(p, stream);
+    case BCNN_ENGINE_LOP3:
+        return launch_conv_lop3(p, stream);
+    case BCNN_ENGINE_MMA_B1:
+        return launch_conv_mma_b1(p, stream);
+    default:
+        return BCNN_ERR_UNSUPPORTED;
+    }
+}
+
+int gemm_problem(ConvProblem &p, const void *A, const void *Wb, const int32_t *thr, void *out,
+                 int64_t M, int N, int K, bool fused)
+{
+    if (M <= 0 || N <= 0 || K <= 0) return BCNN_ERR_INVALID_ARG;
+    if (M >= (1LL << 31)) return BCNN_ERR_UNSUPPORTED;
+    if (K % 32 != 0) return BCNN_ERR_UNSUPPORTED;
+    // a GEMM is the 1x1 convolution over an M x 1 image with K channels
+    return make_conv_problem(p, A, Wb, thr, out, 1, (int)M, 1, K, N, 1, 1, 1, 0, fused);
+}
+
+}  // namespace
+}  // namespace bcnn
+
+using namespace bcnn;
+
+extern "C" {
+
+int bcnn_pack(const float *x, const float *bias, void *out_bits,
+              int B, int H, int W, int C_in, int R, void *stream)
+{
+    if (!x || !out_bits) return BCNN_ERR_INVALID_ARG;
+    if (B <= 0 || H <= 0 || W <= 0 || C_in <= 0 || R <= 0) return BCNN_ERR_INVALID_ARG;
+    const long C = (long)C_in * R;
+    if (C % 32 != 0 || C >= (1L << 24)) return BCNN_ERR_UNSUPPORTED;
+    if (!aligned16(x) || !aligned16(out_bits) || (bias && !aligned16(bias))) return BCNN_ERR_ALIGNMENT;
+    const long npix = (long)B * H * W;
+    if (npix * C >= (1L << 46)) return BCNN_ERR_UNSUPPORTED;
+    return launch_pack(x, bias, static_cast<uint32_t *>(out_bits), npix, C_in, R,
+                       static_cast<cudaStream_t>(stream));
+}
+
+int bcnn_gemm_b1(const void *A_bits, const void *W_bits, int32_t *C, int64_t M, int N, int K, void *stream)
+{
+    return bcnn_gemm_b1_engine(BCNN_ENGINE_AUTO, A_bits, W_bits, nullptr, C, M, N, K, stream);
+}
+
+int bcnn_gemm_b1_fused(const void *A_bits, const void *W_bits, const int32_t *thr, void *out_bits,
+                       int64_t M, int N, int K, void *stream)
+{
+    if (!thr) return BCNN_ERR_INVALID_ARG;
+    return bcnn_gemm_b1_engine(BCNN_ENGINE_AUTO, A_bits, W_bits, thr, out_bits, M, N, K, stream);
+}
+
+int bcnn_conv2d_b1(const void *x_bits, const void *w_bits, int32_t *y, int B, int H, int W, int C_in,
+                   int C_out, int kh, int kw, int stride, int pad, void *stream)
+{
+    return bcnn_conv2d_b1_engine(BCNN_ENGINE_AUTO, x_bits, w_bits, nullptr, y, B, H, W, C_in, C_out,
+                                 kh, kw, stride, pad, stream);
+}
+
+int bcnn_conv2d_b1_fused(const void *x_bits, const void *w_bits, const int32_t *thr, void *y_bits,
+                         int B, int H, int W, int C_in, int C_out, int kh, int kw, int stride, int pad,
+                         void *stream)
+{
+    if (!thr) return BCNN_ERR_INVALID_ARG;
+    return bcnn_conv2d_b1_engine(BCNN_ENGINE_AUTO, x_bits, w_bits, thr, y_bits, B, H, W, C_in, C_out,
+                                 kh, kw, stride, pad, stream);
+}
+
+int bcnn_conv2d_b1_engine(int engine, const void *x_bits, const void *w_bits, const int32_t *thr, void *out,
+                          int B, int H, int W, int C_in, int C_out, int kh, int kw, int stride, int pad,
+                          void *stream)
+{
+    ConvProblem p;
+    const int st = make_conv_problem(p, x_bits, w_bits, thr, out, B, H, W, C_in, C_out, kh, kw, stride, pad,
+                                     thr != nullptr);
+    if (st != BCNN_OK) return st;
+    return dispatch(engine, p, static_cast<cudaStream_t>(stream));
+}
+
+int bcnn_gemm_b1_engine(int engine, const void *A_bits, const void *W_bits, const int32_t *thr, void *out,
+                        int64_t M, int N, int K, void *stream)
+{
+    ConvProblem p;
+    const int st = gemm_problem(p, A_bits, W_bits, thr, out, M, N, K, thr != nullptr);
+    if (st != BCNN_OK) return st;
+    return dispatch(engine, p, static_cast<cudaStream_t>(stream));
+}
+
+int bcnn_device_error(void)
+{
+    int v = 0;
+    if (cudaMemcpyFromSymbol(&v, g_device_error, sizeof(int)) != cudaSuccess) return BCNN_ERR_CUDA;
+    if (v != 0) {
+        const int zero = 0;
+        if (cudaMemcpyToSymbol(g_device_error, &zero, sizeof(int)) != cudaSuccess) return BCNN_ERR_CUDA;
+    }
+    return v;
+}
+
+const char *bcnn_status_string(int status)
+{
+    switch (status) {
+    case BCNN_OK: return "ok";
+    case BCNN_ERR_INVALID_ARG: return "invalid argument";
+    case BCNN_ERR_UNSUPPORTED: return "unsupported shape or engine";
+    case BCNN_ERR_ALIGNMENT: return "pointer not 16-byte aligned";
+    case BCNN_ERR_CUDA: return "CUDA runtime error";
+    default: return status > 0 ? "device-side error code" : "unknown status";
+    }
+}
+
+int bcnn_version(void) { return 100; }
+
+}  // extern "C"

@@ -1,0 +1,48 @@
+// Shared declarations of the CUDA side: problem description handed to every kernel
+// launcher, and small device helpers.
+#pragma once
+#include <cstdint>
+#include <cuda_runtime.h>
+#include "bcnn.h"
+
+namespace bcnn {
+
+// One binary convolution seen as an implicit GEMM: M = B*OH*OW rows, N = C_out
+// columns, K = kh*kw*C_in bits.  A plain GEMM is the 1x1 case with H = M, W = 1.
+struct ConvProblem {
+    const uint32_t *x;   // packed NHWC activations, C_in/32 words per pixel
+    const uint32_t *w;   // packed [C_out][kh][kw][C_in] weights, K/32 words per row
+    const int32_t *thr;  // per-output-channel thresholds, or nullptr for int32 output
+    void *out;           // int32 [M][C_out] or packed bits [M][C_out/32 words]
+    int B, H, W, C_in, C_out, kh, kw, stride, pad, OH, OW;
+    int cw;              // C_in / 32: words per pixel
+    int kwords;          // K / 32
+    int K;               // kh*kw*C_in
+    int M;               // B*OH*OW
+};
+
+// Row m of the implicit patch matrix -> (image, top-left input coordinate).
+struct RowCoord {
+    int b, ih0, iw0;
+};
+
+__device__ __forceinline__ RowCoord row_coord(const ConvProblem &p, int m)
+{
+    RowCoord rc;
+    const int ohw = p.OH * p.OW;
+    rc.b = m / ohw;
+    const int rem = m - rc.b * ohw;
+    const int oh = rem / p.OW;
+    const int ow = rem - oh * p.OW;
+    rc.ih0 = oh * p.stride - p.pad;
+    rc.iw0 = ow * p.stride - p.pad;
+    return rc;
+}
+
+int launch_pack(const float *x, const float *bias, uint32_t *out, long npix, int C_in, int R,
+                cudaStream_t stream);
+int launch_conv_lop3(const ConvProblem &p, cudaStream_t stream);
+int launch_conv_mma_b1(const ConvProblem &p, cudaStream_t stream);
+bool conv_mma_b1_supports(const ConvProblem &p);
+
+}  // namespace bcnn

@@ -1,0 +1,191 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the CPU oracle, bit for bit."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2010_00704_b200 import synth, workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def bk():
+    assert torch.cuda.is_available(), "these tests need a CUDA device"
+    from paper_2010_00704_b200 import build, binding
+    build.build()
+    binding.load()
+    return binding
+
+
+ENGINES = ["auto", "lop3", "mma_b1"]
+
+
+def dev(a):
+    return torch.from_numpy(np.ascontiguousarray(a)).cuda()
+
+
+def guard_alloc(nbytes, dtype=torch.uint8):
+    """Device buffer with 256 guard bytes on both sides, filled with 0xA5."""
+    raw = torch.full((nbytes + 512,), 0xA5, dtype=torch.uint8, device="cuda")
+    return raw, raw[256:256 + nbytes]
+
+
+def check_guards(raw, nbytes):
+    r = raw.cpu().numpy()
+    assert np.all(r[:256] == 0xA5) and np.all(r[256 + nbytes:] == 0xA5), "write outside the output buffer"
+
+
+def run_conv(bk, x, w, thr, stride, pad, engine):
+    """x int8 [B,H,W,Ci] +-1, w int8 [Co,kh,kw,Ci] +-1 -> numpy result (int32 or +-1 int8)."""
+    B, H, W, Ci = x.shape
+    Co, kh, kw, _ = w.shape
+    OH, OW = bk.out_hw(H, W, kh, kw, stride, pad)
+    xb, wb = dev(synth.pack_bits(x)), dev(synth.pack_bits(w))
+    eng = bk.ENGINES[engine]
+    if thr is None:
+        n = B * OH * OW * Co * 4
+        raw, buf = guard_alloc(n)
+        bk.bcnn_conv2d_b1(xb, wb, buf, B, H, W, Ci, Co, kh, kw, stride, pad, engine=eng)
+        torch.cuda.synchronize()
+        check_guards(raw, n)
+        return buf.cpu().numpy().view(np.int32).reshape(B, OH, OW, Co)
+    n = B * OH * OW * Co // 8
+    raw, buf = guard_alloc(n)
+    bk.bcnn_conv2d_b1_fused(xb, wb, dev(thr), buf, B, H, W, Ci, Co, kh, kw, stride, pad, engine=eng)
+    torch.cuda.synchronize()
+    check_guards(raw, n)
+    return synth.unpack_bits(buf.cpu().numpy().reshape(B, OH, OW, Co // 8))
+
+
+CONV_SHAPES = [
+    # B, H, W, Ci, Co, kh, kw, stride, pad
+    (1, 32, 32, 128, 128, 3, 3, 1, 1),     # the single 3x3 workload
+    (2, 9, 13, 32, 64, 3, 3, 1, 1),        # ragged M, one-word pixels
+    (3, 12, 10, 64, 96, 3, 3, 2, 1),       # stride 2, two-word pixels
+    (2, 7, 11, 96, 32, 1, 1, 1, 0),        # 1x1, three-word pixels
+    (1, 17, 5, 32, 160, 3, 1, 2, 0),       # kh != kw, ragged N tile
+    (2, 6, 9, 160, 224, 1, 3, 1, 2),       # pad larger than needed, wide N
+    (1, 40, 40, 256, 256, 3, 3, 2, 1),     # several M and N tiles, K = 2304
+    (5, 14, 14, 512, 64, 3, 3, 1, 1),      # K = 4608
+    (1, 3, 3, 32, 32, 5, 5, 1, 2),         # kernel larger than the image interior
+]
+
+
+@pytest.mark.parametrize("engine", ENGINES)
+@pytest.mark.parametrize("shape", CONV_SHAPES)
+def test_conv_int32_and_fused(bk, oracle, shape, engine):
+    B, H, W, Ci, Co, kh, kw, s, p = shape
+    rng = np.random.default_rng(900 + sum(shape))
+    x = synth.pm1(rng, (B, H, W, Ci))
+    w = synth.pm1(rng, (Co, kh, kw, Ci))
+    want = oracle.conv2d(x, w, s, p)
+    got = run_conv(bk, x, w, None, s, p, engine)
+    assert np.array_equal(got, want)
+    K = kh * kw * Ci
+    thr = synth.thresholds(rng, K, Co)
+    thr[::3] = want.reshape(-1, Co)[0, ::3]           # exact ties on some channels
+    got_bits = run_conv(bk, x, w, thr, s, p, engine)
+    assert np.array_equal(got_bits, oracle.threshold(want, thr))
+
+
+@pytest.mark.parametrize("engine", ENGINES)
+def test_conv_int32_any_channel_count(bk, oracle, engine):
+    # int32 output accepts C_out that is not a multiple of 32 (or even)
+    for Co in (1, 7, 30, 33):
+        rng = np.random.default_rng(50 + Co)
+        x = synth.pm1(rng, (1, 6, 7, 64))
+        w = synth.pm1(rng, (Co, 3, 3, 64))
+        assert np.array_equal(run_conv(bk, x, w, None, 1, 1, engine), oracle.conv2d(x, w, 1, 1))
+
+
+@pytest.mark.parametrize("engine", ENGINES)
+def test_conv_constant_inputs(bk, engine):
+    # closed forms straight on the GPU: all -1 activations -> -+K everywhere, borders included
+    B, H, W, Ci, Co = 1, 9, 9, 64, 32
+    K = 9 * Ci
+    xm = -np.ones((B, H, W, Ci), np.int8)
+    wp = np.ones((Co, 3, 3, Ci), np.int8)
+    assert np.all(run_conv(bk, xm, wp, None, 1, 1, engine) == -K)
+    assert np.all(run_conv(bk, xm, -wp, None, 2, 1, engine) == K)
+    y = run_conv(bk, -xm, wp, None, 1, 1, engine)[0, :, :, 0]
+    assert y[4, 4] == K and y[0, 4] == K - 6 * Ci and y[0, 0] == K - 10 * Ci
+
+
+GEMM_SHAPES = [(1024, 1024, 512), (1024, 1024, 2304), (300, 200, 96), (129, 33, 1056), (64, 512, 4608), (1, 32, 32)]
+
+
+@pytest.mark.parametrize("engine", ENGINES)
+@pytest.mark.parametrize("shape", GEMM_SHAPES)
+def test_gemm_int32_and_fused(bk, oracle, shape, engine):
+    M, N, K = shape
+    rng = np.random.default_rng(1000 + sum(shape))
+    A = synth.pm1(rng, (M, K))
+    Wt = synth.pm1(rng, (N, K))
+    want = oracle.gemm(A, Wt)
+    Ab, Wb = dev(synth.pack_bits(A)), dev(synth.pack_bits(Wt))
+    raw, C = guard_alloc(M * N * 4)
+    bk.bcnn_gemm_b1(Ab, Wb, C, M, N, K, engine=bk.ENGINES[engine])
+    torch.cuda.synchronize()
+    check_guards(raw, M * N * 4)
+    assert np.array_equal(C.cpu().numpy().view(np.int32).reshape(M, N), want)
+    if N % 32 == 0:
+        thr = synth.thresholds(rng, K, N)
+        raw, ob = guard_alloc(M * N // 8)
+        bk.bcnn_gemm_b1_fused(Ab, Wb, dev(thr), ob, M, N, K, engine=bk.ENGINES[engine])
+        torch.cuda.synchronize()
+        check_guards(raw, M * N // 8)
+        assert np.array_equal(synth.unpack_bits(ob.cpu().numpy().reshape(M, N // 8)), oracle.threshold(want, thr))
+
+
+PACK_SHAPES = [
+    # B, H, W, C_in, R, bias
+    (2, 5, 7, 32, 1, False), (2, 5, 7, 64, 1, True), (1, 33, 9, 96, 1, True), (3, 8, 8, 4, 8, True),
+    (3, 8, 8, 4, 8, False), (1, 4, 5, 8, 4, True), (2, 3, 3, 16, 6, True), (1, 2, 2, 3, 32, True),
+    (1, 64, 64, 128, 1, True),
+]
+
+
+@pytest.mark.parametrize("shape", PACK_SHAPES)
+def test_pack(bk, oracle, shape):
+    B, H, W, Ci, R, has_bias = shape
+    rng = np.random.default_rng(300 + sum(shape[:5]))
+    x = synth.real_input(rng, (B, H, W, Ci))
+    C = Ci * R
+    bias = synth.real_input(rng, (C,)) if has_bias else None
+    # plant ties and special values
+    flat = x.reshape(-1)
+    flat[:8] = [0.0, -0.0, np.inf, -np.inf, np.nan, 1e-45, -1e-45, 0.0]
+    if has_bias:
+        flat[8] = -bias[8 % Ci] if R == 1 else flat[8]
+    want = oracle.binarize(x, bias, R)
+    n = B * H * W * C // 8
+    raw, out = guard_alloc(n)
+    bk.bcnn_pack(dev(x), None if bias is None else dev(bias), out, B, H, W, Ci, R)
+    torch.cuda.synchronize()
+    check_guards(raw, n)
+    assert np.array_equal(synth.unpack_bits(out.cpu().numpy().reshape(B, H, W, C // 8)), want)
+
+
+def test_pack_weights_layout(bk, oracle):
+    # packing real weights [C_out][kh][kw][C_in] with the same call gives the conv weight layout
+    rng = np.random.default_rng(77)
+    wr = synth.real_input(rng, (64, 3, 3, 32))
+    out = torch.empty(64 * 9 * 32 // 8, dtype=torch.uint8, device="cuda")
+    bk.bcnn_pack(dev(wr), None, out, 64, 3, 3, 32, 1)
+    torch.cuda.synchronize()
+    assert np.array_equal(out.cpu().numpy().reshape(64, 3, 3, 4), synth.pack_bits(oracle.sign_weights(wr)))
+
+
+def test_errors_launch_nothing(bk):
+    a = torch.zeros(4096, dtype=torch.uint8, device="cuda")
+    with pytest.raises(bk.BcnnError) as e:
+        bk.bcnn_conv2d_b1(a, a, a, 1, 4, 4, 48, 32, 3, 3, 1, 1)
+    assert e.value.status == -2
+    with pytest.raises(bk.BcnnError) as e:
+        bk.bcnn_gemm_b1(a[4:], a, a, 8, 8, 32)
+    assert e.value.status == -3
+    with pytest.raises(bk.BcnnError):
+        bk.bcnn_gemm_b1_fused(a, a, None, a, 8, 32, 32)
+    torch.cuda.synchronize()
+    assert int(a.sum()) == 0
+    assert bk.bcnn_device_error() == 0
