@@ -341,8 +341,95 @@ def run_gpu(args):
     return 0
 
 
+def run_sweep(args):
+    """Engine comparison on the GEMM sweep and the single-layer workloads (not the headline line).
+
+    Prints one JSON object per (shape, output kind, engine): time (median of --steps launches after
+    --warmup), TOPS and, for the int32 output, the output write rate."""
+    import torch
+    from paper_2010_00704_b200 import build, binding
+    build.build()
+    binding.load()
+    torch.cuda.set_device(0)
+    engines = args.engines.split(",")
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+
+    def timeit(fn):
+        for _ in range(args.warmup):
+            fn()
+        ts = []
+        for _ in range(args.steps):
+            flush.zero_()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            fn()
+            b.record()
+            torch.cuda.synchronize()
+            ts.append(a.elapsed_time(b))
+        return float(np.median(ts)), float(min(ts))
+
+    rows = []
+    rng = np.random.default_rng(1)
+    shapes = []
+    if args.sweep_set in ("gemm", "all"):
+        for mn in wl.GEMM_SWEEP_MN:
+            for k in wl.GEMM_SWEEP_K:
+                shapes.append(("gemm", mn, mn, k, None, 1))
+    if args.sweep_set in ("conv", "all"):
+        shapes.append(("conv", None, None, None, wl.SINGLE_3X3, wl.SINGLE_3X3_BATCH))
+        for l in wl.STEM_DOWN:
+            shapes.append(("conv", None, None, None, l, wl.STEM_DOWN_BATCH))
+        for l in wl.BLOCK_STACK:
+            shapes.append(("conv", None, None, None, l, wl.BLOCK_STACK_BATCH))
+        for l in wl.BACKBONE18:
+            shapes.append(("conv", None, None, None, l, wl.BACKBONE18_BATCH))
+    for kind, M, N, K, l, B in shapes:
+        if kind == "gemm":
+            A = torch.from_numpy(synth.random_bits(rng, (M, K // 8))).cuda()
+            Wb = torch.from_numpy(synth.random_bits(rng, (N, K // 8))).cuda()
+            thr = torch.from_numpy(synth.thresholds(rng, K, N)).cuda()
+            out32 = torch.empty(M * N, dtype=torch.int32, device="cuda")
+            outb = torch.empty(M * N // 8, dtype=torch.uint8, device="cuda")
+            ops = wl.gemm_ops(M, N, K)
+            name = f"gemm M=N={M} K={K}"
+            calls = {
+                "int32": lambda e: binding.bcnn_gemm_b1(A, Wb, out32, M, N, K, engine=e),
+                "fused": lambda e: binding.bcnn_gemm_b1_fused(A, Wb, thr, outb, M, N, K, engine=e),
+            }
+            out_bytes = {"int32": 4 * M * N, "fused": M * N // 8}
+        else:
+            x = torch.from_numpy(synth.random_bits(rng, (l.in_bytes(B),))).cuda()
+            Wb = torch.from_numpy(synth.random_bits(rng, (l.w_bytes(),))).cuda()
+            thr = torch.from_numpy(synth.thresholds(rng, l.K, l.C_out)).cuda()
+            outb = torch.empty(l.out_bits_bytes(B), dtype=torch.uint8, device="cuda")
+            ops = l.ops(B)
+            name = f"conv {l.name} B={B} M={l.M(B)} N={l.C_out} K={l.K}"
+            calls = {
+                "fused": lambda e: binding.bcnn_conv2d_b1_fused(x, Wb, thr, outb, B, l.H, l.W, l.C_in, l.C_out,
+                                                                 l.k, l.k, l.stride, l.pad, engine=e),
+            }
+            out_bytes = {"fused": l.out_bits_bytes(B)}
+        for okind, call in calls.items():
+            for en in engines:
+                e = binding.ENGINES[en]
+                try:
+                    med, mn_ = timeit(lambda: call(e))
+                except binding.BcnnError as ex:
+                    rows.append({"shape": name, "out": okind, "engine": en, "error": str(ex)})
+                    continue
+                rows.append({"shape": name, "out": okind, "engine": en, "ms": med, "ms_min": mn_,
+                             "tops": ops / (med / 1e3) / 1e12, "out_gbs": out_bytes[okind] / (med / 1e3) / 1e9})
+                print(json.dumps(rows[-1]), flush=True)
+    err = binding.bcnn_device_error()
+    print(json.dumps({"device_error": err}))
+    return 0 if err == 0 else 1
+
+
 def main():
     ap = argparse.ArgumentParser()
+    ap.add_argument("--mode", default="bench", choices=["bench", "sweep"])
+    ap.add_argument("--engines", default="auto,lop3,mma_b1,tc_i8")
+    ap.add_argument("--sweep-set", default="all", choices=["gemm", "conv", "all"])
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=5)
@@ -351,6 +438,8 @@ def main():
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)
+    if args.mode == "sweep":
+        return run_sweep(args)
     return run_gpu(args)
 
 

@@ -19,7 +19,16 @@ struct ConvProblem {
     int kwords;          // K / 32
     int K;               // kh*kw*C_in
     int M;               // B*OH*OW
+    uint32_t cw_magic;   // floor(2^32 / cw) + 1 (0 when cw == 1): n / cw == umulhi(n, magic) for n*cw < 2^32
+    uint32_t kw_magic;   // same for the kernel width kw
+    int *err;            // device error word (bounded waits report here)
 };
+
+// n / d through a precomputed multiplier (exact while n * d < 2^32); magic == 0 encodes d == 1.
+__device__ __forceinline__ int fast_div(int n, uint32_t magic)
+{
+    return magic ? (int)__umulhi((uint32_t)n, magic) : n;
+}
 
 // Row m of the implicit patch matrix -> (image, top-left input coordinate).
 struct RowCoord {
@@ -44,5 +53,8 @@ int launch_pack(const float *x, const float *bias, uint32_t *out, long npix, int
 int launch_conv_lop3(const ConvProblem &p, cudaStream_t stream);
 int launch_conv_mma_b1(const ConvProblem &p, cudaStream_t stream);
 bool conv_mma_b1_supports(const ConvProblem &p);
+int launch_conv_tc_i8(const ConvProblem &p, cudaStream_t stream);
+bool conv_tc_i8_supports(const ConvProblem &p);
+int *device_error_word();   // device address of the error word of the current device (nullptr on failure)
 
 }  // namespace bcnn

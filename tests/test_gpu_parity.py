@@ -17,7 +17,7 @@ def bk():
     return binding
 
 
-ENGINES = ["auto", "lop3", "mma_b1"]
+ENGINES = ["auto", "lop3", "mma_b1", "tc_i8"]
 
 
 def dev(a):
