@@ -384,6 +384,9 @@ def run_sweep(args):
         for l in wl.BACKBONE18:
             shapes.append(("conv", None, None, None, l, wl.BACKBONE18_BATCH))
     for kind, M, N, K, l, B in shapes:
+        label = f"gemm M=N={M} K={K}" if kind == "gemm" else f"conv {l.name} "
+        if args.only and args.only not in label:
+            continue
         if kind == "gemm":
             A = torch.from_numpy(synth.random_bits(rng, (M, K // 8))).cuda()
             Wb = torch.from_numpy(synth.random_bits(rng, (N, K // 8))).cuda()
@@ -410,6 +413,8 @@ def run_sweep(args):
             }
             out_bytes = {"fused": l.out_bits_bytes(B)}
         for okind, call in calls.items():
+            if okind not in args.outs.split(","):
+                continue
             for en in engines:
                 e = binding.ENGINES[en]
                 try:
@@ -428,8 +433,10 @@ def run_sweep(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--mode", default="bench", choices=["bench", "sweep"])
-    ap.add_argument("--engines", default="auto,lop3,mma_b1,tc_i8")
+    ap.add_argument("--engines", default="auto,lop3,mma_b1,tc_i8,mma_s8")
     ap.add_argument("--sweep-set", default="all", choices=["gemm", "conv", "all"])
+    ap.add_argument("--only", default="", help="sweep mode: run only shapes whose label contains this text")
+    ap.add_argument("--outs", default="int32,fused", help="sweep mode: output kinds to run")
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=5)

@@ -72,6 +72,8 @@ int dispatch(int engine, const ConvProblem &p, cudaStream_t stream)
         return launch_conv_mma_b1(p, stream);
     case BCNN_ENGINE_TC_I8:
         return launch_conv_tc_i8(p, stream);
+    case BCNN_ENGINE_MMA_S8:
+        return launch_conv_mma_s8(p, stream);
     default:
         return BCNN_ERR_UNSUPPORTED;
     }

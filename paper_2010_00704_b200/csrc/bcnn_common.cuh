@@ -53,6 +53,8 @@ int launch_pack(const float *x, const float *bias, uint32_t *out, long npix, int
 int launch_conv_lop3(const ConvProblem &p, cudaStream_t stream);
 int launch_conv_mma_b1(const ConvProblem &p, cudaStream_t stream);
 bool conv_mma_b1_supports(const ConvProblem &p);
+int launch_conv_mma_s8(const ConvProblem &p, cudaStream_t stream);
+bool conv_mma_s8_supports(const ConvProblem &p);
 int launch_conv_tc_i8(const ConvProblem &p, cudaStream_t stream);
 bool conv_tc_i8_supports(const ConvProblem &p);
 int *device_error_word();   // device address of the error word of the current device (nullptr on failure)

@@ -17,7 +17,7 @@ def bk():
     return binding
 
 
-ENGINES = ["auto", "lop3", "mma_b1", "tc_i8"]
+ENGINES = ["auto", "lop3", "mma_b1", "tc_i8", "mma_s8"]
 
 
 def dev(a):
@@ -35,6 +35,16 @@ def check_guards(raw, nbytes):
     assert np.all(r[:256] == 0xA5) and np.all(r[256 + nbytes:] == 0xA5), "write outside the output buffer"
 
 
+def call_or_skip(bk, engine, fn):
+    """An explicitly chosen engine may decline a shape (BCNN_ERR_UNSUPPORTED); "auto" may not."""
+    try:
+        fn()
+    except bk.BcnnError as e:
+        if e.status == -2 and engine != "auto":
+            pytest.skip(f"engine {engine} does not take this shape")
+        raise
+
+
 def run_conv(bk, x, w, thr, stride, pad, engine):
     """x int8 [B,H,W,Ci] +-1, w int8 [Co,kh,kw,Ci] +-1 -> numpy result (int32 or +-1 int8)."""
     B, H, W, Ci = x.shape
@@ -45,13 +55,13 @@ def run_conv(bk, x, w, thr, stride, pad, engine):
     if thr is None:
         n = B * OH * OW * Co * 4
         raw, buf = guard_alloc(n)
-        bk.bcnn_conv2d_b1(xb, wb, buf, B, H, W, Ci, Co, kh, kw, stride, pad, engine=eng)
+        call_or_skip(bk, engine, lambda: bk.bcnn_conv2d_b1(xb, wb, buf, B, H, W, Ci, Co, kh, kw, stride, pad, engine=eng))
         torch.cuda.synchronize()
         check_guards(raw, n)
         return buf.cpu().numpy().view(np.int32).reshape(B, OH, OW, Co)
     n = B * OH * OW * Co // 8
     raw, buf = guard_alloc(n)
-    bk.bcnn_conv2d_b1_fused(xb, wb, dev(thr), buf, B, H, W, Ci, Co, kh, kw, stride, pad, engine=eng)
+    call_or_skip(bk, engine, lambda: bk.bcnn_conv2d_b1_fused(xb, wb, dev(thr), buf, B, H, W, Ci, Co, kh, kw, stride, pad, engine=eng))
     torch.cuda.synchronize()
     check_guards(raw, n)
     return synth.unpack_bits(buf.cpu().numpy().reshape(B, OH, OW, Co // 8))
@@ -124,14 +134,14 @@ def test_gemm_int32_and_fused(bk, oracle, shape, engine):
     want = oracle.gemm(A, Wt)
     Ab, Wb = dev(synth.pack_bits(A)), dev(synth.pack_bits(Wt))
     raw, C = guard_alloc(M * N * 4)
-    bk.bcnn_gemm_b1(Ab, Wb, C, M, N, K, engine=bk.ENGINES[engine])
+    call_or_skip(bk, engine, lambda: bk.bcnn_gemm_b1(Ab, Wb, C, M, N, K, engine=bk.ENGINES[engine]))
     torch.cuda.synchronize()
     check_guards(raw, M * N * 4)
     assert np.array_equal(C.cpu().numpy().view(np.int32).reshape(M, N), want)
     if N % 32 == 0:
         thr = synth.thresholds(rng, K, N)
         raw, ob = guard_alloc(M * N // 8)
-        bk.bcnn_gemm_b1_fused(Ab, Wb, dev(thr), ob, M, N, K, engine=bk.ENGINES[engine])
+        call_or_skip(bk, engine, lambda: bk.bcnn_gemm_b1_fused(Ab, Wb, dev(thr), ob, M, N, K, engine=bk.ENGINES[engine]))
         torch.cuda.synchronize()
         check_guards(raw, M * N // 8)
         assert np.array_equal(synth.unpack_bits(ob.cpu().numpy().reshape(M, N // 8)), oracle.threshold(want, thr))
