@@ -21,6 +21,16 @@ int *device_error_word()
 
 namespace {
 
+// (mul, shift) of exact_div for the divisor d >= 1
+void exact_div_params(uint32_t d, uint32_t &mul, uint32_t &shift)
+{
+    if (d <= 1) { mul = 0; shift = 0; return; }
+    uint32_t s = 0;
+    while ((1ULL << s) < d) ++s;
+    mul = (uint32_t)(((1ULL << 32) * ((1ULL << s) - d)) / d + 1);
+    shift = s;
+}
+
 inline bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 int make_conv_problem(ConvProblem &p, const void *x, const void *w, const int32_t *thr, void *out,
@@ -53,6 +63,8 @@ int make_conv_problem(ConvProblem &p, const void *x, const void *w, const int32_
     p.M = (int)M;
     p.cw_magic = p.cw == 1 ? 0u : (uint32_t)((1ULL << 32) / (uint64_t)p.cw) + 1u;
     p.err = nullptr;
+    exact_div_params((uint32_t)OW, p.ow_mul, p.ow_shift);
+    exact_div_params((uint32_t)(OH * OW), p.ohw_mul, p.ohw_shift);
     p.kw_magic = kw == 1 ? 0u : (uint32_t)((1ULL << 32) / (uint64_t)kw) + 1u;
     return BCNN_OK;
 }
@@ -61,9 +73,11 @@ int dispatch(int engine, const ConvProblem &p, cudaStream_t stream)
 {
     switch (engine) {
     case BCNN_ENGINE_AUTO:
-        // Measured on B200: the tcgen05 int8 engine wins everywhere except the narrow
-        // (C_out <= 32) layers, where its 128 x 64 tile is mostly padding.
-        if (p.C_out > 32 && conv_tc_i8_supports(p)) return launch_conv_tc_i8(p, stream);
+        // Measured on B200 (bench.py --mode sweep): the tcgen05 engine wins from 128 output
+        // channels up, the register-fed warp-level int8 engine on the narrow layers; the
+        // single-bit mma.sync and CUDA-core engines never win and serve as fallbacks.
+        if (p.C_out <= 64 && conv_mma_s8_supports(p)) return launch_conv_mma_s8(p, stream);
+        if (conv_tc_i8_supports(p)) return launch_conv_tc_i8(p, stream);
         if (conv_mma_b1_supports(p)) return launch_conv_mma_b1(p, stream);
         return launch_conv_lop3(p, stream);
     case BCNN_ENGINE_LOP3:

@@ -22,7 +22,19 @@ struct ConvProblem {
     uint32_t cw_magic;   // floor(2^32 / cw) + 1 (0 when cw == 1): n / cw == umulhi(n, magic) for n*cw < 2^32
     uint32_t kw_magic;   // same for the kernel width kw
     int *err;            // device error word (bounded waits report here)
+    uint32_t ow_mul, ow_shift;    // exact division of any 32-bit value by OW      (see exact_div)
+    uint32_t ohw_mul, ohw_shift;  // exact division of any 32-bit value by OH * OW
 };
+
+// Exact n / d for every 32-bit n with a precomputed (mul, shift) pair: with s = ceil(log2 d) and
+// mul = floor(2^32 * (2^s - d) / d) + 1,  n / d = (t + ((n - t) >> 1)) >> (s - 1),  t = umulhi(n, mul).
+// d == 1 is encoded as shift == 0.
+__device__ __forceinline__ uint32_t exact_div(uint32_t n, uint32_t mul, uint32_t shift)
+{
+    if (shift == 0) return n;
+    const uint32_t t = __umulhi(n, mul);
+    return (t + ((n - t) >> 1)) >> (shift - 1);
+}
 
 // n / d through a precomputed multiplier (exact while n * d < 2^32); magic == 0 encodes d == 1.
 __device__ __forceinline__ int fast_div(int n, uint32_t magic)
@@ -39,9 +51,9 @@ __device__ __forceinline__ RowCoord row_coord(const ConvProblem &p, int m)
 {
     RowCoord rc;
     const int ohw = p.OH * p.OW;
-    rc.b = m / ohw;
+    rc.b = (int)exact_div((uint32_t)m, p.ohw_mul, p.ohw_shift);
     const int rem = m - rc.b * ohw;
-    const int oh = rem / p.OW;
+    const int oh = (int)exact_div((uint32_t)rem, p.ow_mul, p.ow_shift);
     const int ow = rem - oh * p.OW;
     rc.ih0 = oh * p.stride - p.pad;
     rc.iw0 = ow * p.stride - p.pad;

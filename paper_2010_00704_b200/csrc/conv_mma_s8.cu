@@ -32,7 +32,7 @@ __device__ __forceinline__ void mma_u8(int (&d)[4], uint32_t a0, uint32_t a1, ui
 }
 
 template <int NA, bool FUSED>
-__global__ void __launch_bounds__(THREADS)
+__global__ void __launch_bounds__(THREADS, 2)
 conv_mma_s8_kernel(const ConvProblem p)
 {
     constexpr int BN = 8 * NA;
@@ -107,9 +107,9 @@ conv_mma_s8_kernel(const ConvProblem p)
                 for (int e = 0; e < 4; ++e) acc[a][j][e] = 0;
         }
 
-        int r = 0, t = 0, cj = 0;      // tap and channel word of the current K word (warp-uniform)
-        for (int kw = 0; kw < p.kwords; ++kw) {
-            uint32_t w[MA][2];
+        // K loop, software-pipelined: the words of step kw+1 are in flight while step kw is multiplied
+        int r = 0, t = 0, cj = 0;      // tap and channel word of the K word being loaded (warp-uniform)
+        auto load_words = [&](uint32_t (&w)[MA][2]) {
 #pragma unroll
             for (int a = 0; a < MA; ++a)
 #pragma unroll
@@ -119,9 +119,22 @@ conv_mma_s8_kernel(const ConvProblem p)
                     if (ok[a][h] && ih >= 0 && ih < p.H && iw >= 0 && iw < p.W)
                         v = __ldg(xb[a][h] + ((long)ih * p.W + iw) * p.cw + cj);
                     w[a][h] = v;
-                    pa[a][h] += __popc(v);
                 }
+            if (++cj == p.cw) {
+                cj = 0;
+                if (++t == p.kw) { t = 0; ++r; }
+            }
+        };
+        uint32_t w[MA][2], wn[MA][2];
+        load_words(w);
+        for (int kw = 0; kw < p.kwords; ++kw) {
+            if (kw + 1 < p.kwords) load_words(wn);
             const uint2 *wf = wfrag + (size_t)kw * NA * 32 + lane;
+#pragma unroll
+            for (int a = 0; a < MA; ++a) {
+                pa[a][0] += __popc(w[a][0]);
+                pa[a][1] += __popc(w[a][1]);
+            }
 #pragma unroll
             for (int j = 0; j < NA; ++j) {
                 const uint2 b = wf[j * 32];
@@ -129,9 +142,10 @@ conv_mma_s8_kernel(const ConvProblem p)
                 for (int a = 0; a < MA; ++a)
                     mma_u8(acc[a][j], w[a][0] & mlo, w[a][1] & mlo, w[a][0] & mhi, w[a][1] & mhi, b);
             }
-            if (++cj == p.cw) {
-                cj = 0;
-                if (++t == p.kw) { t = 0; ++r; }
+#pragma unroll
+            for (int a = 0; a < MA; ++a) {
+                w[a][0] = wn[a][0];
+                w[a][1] = wn[a][1];
             }
         }
 
@@ -191,25 +205,20 @@ int launch_na(const ConvProblem &p, cudaStream_t stream)
     cudaGetDevice(&dev);
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     const long nblocks = ((long)p.M + 16 * MA - 1) / (16 * MA);
-    const int per_sm = smem > 100 * 1024 ? 1 : (smem > 48 * 1024 ? 2 : 3);
+    void (*k)(const ConvProblem) = p.thr ? conv_mma_s8_kernel<NA, true> : conv_mma_s8_kernel<NA, false>;
+    if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return BCNN_ERR_CUDA;
+    int per_sm = 1;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k, THREADS, smem) != cudaSuccess || per_sm < 1) per_sm = 1;
+    // persistent grid: every resident CTA slot of the chip, split over the N tiles
+    const long ny = (p.C_out + 8 * NA - 1) / (8 * NA);
+    if (ny > 65535) return BCNN_ERR_UNSUPPORTED;
     long gx = (nblocks + THREADS / 32 - 1) / (THREADS / 32);
-    const long cap = (long)sms * per_sm;
+    long cap = ((long)sms * per_sm) / ny;
+    if (cap < 1) cap = 1;
     if (gx > cap) gx = cap;
     if (gx < 1) gx = 1;
-    dim3 grid((unsigned)gx, (p.C_out + 8 * NA - 1) / (8 * NA));
-    if (grid.y > 65535) return BCNN_ERR_UNSUPPORTED;
-    cudaError_t e;
-    if (p.thr) {
-        auto k = conv_mma_s8_kernel<NA, true>;
-        e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e != cudaSuccess) return BCNN_ERR_CUDA;
-        k<<<grid, THREADS, smem, stream>>>(p);
-    } else {
-        auto k = conv_mma_s8_kernel<NA, false>;
-        e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
-        if (e != cudaSuccess) return BCNN_ERR_CUDA;
-        k<<<grid, THREADS, smem, stream>>>(p);
-    }
+    dim3 grid((unsigned)gx, (unsigned)ny);
+    k<<<grid, THREADS, smem, stream>>>(p);
     return cudaGetLastError() == cudaSuccess ? BCNN_OK : BCNN_ERR_CUDA;
 }
 

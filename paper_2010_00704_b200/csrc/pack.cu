@@ -73,20 +73,33 @@ __global__ void __launch_bounds__(256)
 pack_c4r8_kernel(const float4 *__restrict__ x, const float *__restrict__ bias,
                  uint32_t *__restrict__ out, long npix)
 {
+    constexpr int U = 4;                       // pixels in flight per thread
     __shared__ float sb[32];
     if (threadIdx.x < 32) sb[threadIdx.x] = bias ? bias[threadIdx.x] : 0.0f;
     __syncthreads();
-    const long stride = (long)gridDim.x * blockDim.x;
-    for (long p = (long)blockIdx.x * blockDim.x + threadIdx.x; p < npix; p += stride) {
-        const float4 v = __ldcs(x + p);
-        const float f[4] = {v.x, v.y, v.z, v.w};
-        uint32_t word = 0;
+    float b[32];
 #pragma unroll
-        for (int c = 0; c < 32; ++c) {
-            const float s = bias ? __fadd_rn(f[c & 3], sb[c]) : f[c & 3];
-            word |= (s >= 0.0f ? 1u : 0u) << c;
+    for (int c = 0; c < 32; ++c) b[c] = sb[c];
+    const long stride = (long)gridDim.x * blockDim.x;
+    for (long p0 = (long)blockIdx.x * blockDim.x + threadIdx.x; p0 < npix; p0 += stride * U) {
+        float4 v[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const long p = p0 + u * stride;
+            v[u] = (p < npix) ? __ldcs(x + p) : make_float4(0.f, 0.f, 0.f, 0.f);
         }
-        out[p] = word;
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const long p = p0 + u * stride;
+            const float f[4] = {v[u].x, v[u].y, v[u].z, v[u].w};
+            uint32_t word = 0;
+#pragma unroll
+            for (int c = 0; c < 32; ++c) {
+                const float s = bias ? __fadd_rn(f[c & 3], b[c]) : f[c & 3];
+                word |= (s >= 0.0f ? 1u : 0u) << c;
+            }
+            if (p < npix) __stcs(out + p, word);
+        }
     }
 }
 
@@ -112,9 +125,10 @@ int launch_pack(const float *x, const float *bias, uint32_t *out, long npix, int
         else
             pack_stream_kernel<UNROLL, false><<<(int)blocks, threads, 0, stream>>>(x, bias, out, nwords, cwords);
     } else if (C_in == 4 && R == 8) {
-        long blocks = (npix + threads - 1) / threads;
-        const long cap = (long)sms * 8;
+        long blocks = (npix + threads * 4 - 1) / (threads * 4);
+        const long cap = (long)sms * 6;
         if (blocks > cap) blocks = cap;
+        if (blocks < 1) blocks = 1;
         pack_c4r8_kernel<<<(int)blocks, threads, 0, stream>>>(reinterpret_cast<const float4 *>(x), bias, out, npix);
     } else {
         long blocks = (nwords + 7) / 8;
