@@ -126,6 +126,13 @@ int bcnn_gemm_b1_engine(int engine, const void *A_bits, const void *W_bits, cons
                         void *out, int64_t M, int N, int K, void *stream);
 
 /*
+ * Which engine BCNN_ENGINE_AUTO runs for a convolution of this shape (fused != 0: the packed
+ * output).  Returns a bcnn_engine value, or a negative bcnn_status for an invalid shape.
+ * No pointers, no launch.  A GEMM is the shape (1, M, 1, K, N, 1, 1, 1, 0).
+ */
+int bcnn_auto_engine(int B, int H, int W, int C_in, int C_out, int kh, int kw, int stride, int pad, int fused);
+
+/*
  * Device-side error word.  Kernels that wait on hardware barriers give up after a
  * bounded number of polls and record a non-zero code here instead of hanging.
  * Reads the word of the current device (synchronises that device) and clears it.

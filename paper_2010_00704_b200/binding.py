@@ -21,7 +21,7 @@ ENGINES = {"auto": ENGINE_AUTO, "lop3": ENGINE_LOP3, "mma_b1": ENGINE_MMA_B1, "t
 
 EXPORTS = (
     "bcnn_pack", "bcnn_gemm_b1", "bcnn_gemm_b1_fused", "bcnn_conv2d_b1", "bcnn_conv2d_b1_fused",
-    "bcnn_conv2d_b1_engine", "bcnn_gemm_b1_engine", "bcnn_device_error", "bcnn_status_string",
+    "bcnn_conv2d_b1_engine", "bcnn_gemm_b1_engine", "bcnn_auto_engine", "bcnn_device_error", "bcnn_status_string",
     "bcnn_version",
 )
 
@@ -49,6 +49,7 @@ def load() -> ctypes.CDLL:
         lib.bcnn_conv2d_b1_fused.argtypes = [vp, vp, vp, vp] + [i32] * 9 + [vp]
         lib.bcnn_conv2d_b1_engine.argtypes = [i32, vp, vp, vp, vp] + [i32] * 9 + [vp]
         lib.bcnn_gemm_b1_engine.argtypes = [i32, vp, vp, vp, vp, i64, i32, i32, vp]
+        lib.bcnn_auto_engine.argtypes = [i32] * 10
         lib.bcnn_device_error.argtypes = []
         lib.bcnn_status_string.argtypes = [i32]
         lib.bcnn_status_string.restype = ctypes.c_char_p
@@ -117,6 +118,14 @@ def bcnn_conv2d_b1_fused(x_bits, w_bits, thr, y_bits, B, H, W, C_in, C_out, kh, 
     _check(load().bcnn_conv2d_b1_engine(engine, _p(x_bits), _p(w_bits), _p(thr), _p(y_bits), B, H, W, C_in,
                                         C_out, kh, kw, stride, pad, _stream()), "bcnn_conv2d_b1_fused")
     return y_bits
+
+
+def bcnn_auto_engine(B, H, W, C_in, C_out, kh, kw, stride, pad, fused=True) -> str:
+    """Name of the engine BCNN_ENGINE_AUTO picks for this shape."""
+    e = load().bcnn_auto_engine(B, H, W, C_in, C_out, kh, kw, stride, pad, 1 if fused else 0)
+    if e < 0:
+        raise BcnnError(e, "bcnn_auto_engine")
+    return {v: k for k, v in ENGINES.items()}[e]
 
 
 def bcnn_device_error() -> int:

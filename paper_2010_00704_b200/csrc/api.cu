@@ -69,17 +69,21 @@ int make_conv_problem(ConvProblem &p, const void *x, const void *w, const int32_
     return BCNN_OK;
 }
 
+// Measured on B200 (bench.py --mode sweep): the tcgen05 engine wins from 128 output channels
+// up, the register-fed warp-level int8 engine on the narrow layers; the single-bit mma.sync
+// and CUDA-core engines never win and serve as fallbacks.
+int auto_engine(const ConvProblem &p)
+{
+    if (p.C_out <= 64 && conv_mma_s8_supports(p)) return BCNN_ENGINE_MMA_S8;
+    if (conv_tc_i8_supports(p)) return BCNN_ENGINE_TC_I8;
+    if (conv_mma_b1_supports(p)) return BCNN_ENGINE_MMA_B1;
+    return BCNN_ENGINE_LOP3;
+}
+
 int dispatch(int engine, const ConvProblem &p, cudaStream_t stream)
 {
+    if (engine == BCNN_ENGINE_AUTO) engine = auto_engine(p);
     switch (engine) {
-    case BCNN_ENGINE_AUTO:
-        // Measured on B200 (bench.py --mode sweep): the tcgen05 engine wins from 128 output
-        // channels up, the register-fed warp-level int8 engine on the narrow layers; the
-        // single-bit mma.sync and CUDA-core engines never win and serve as fallbacks.
-        if (p.C_out <= 64 && conv_mma_s8_supports(p)) return launch_conv_mma_s8(p, stream);
-        if (conv_tc_i8_supports(p)) return launch_conv_tc_i8(p, stream);
-        if (conv_mma_b1_supports(p)) return launch_conv_mma_b1(p, stream);
-        return launch_conv_lop3(p, stream);
     case BCNN_ENGINE_LOP3:
         return launch_conv_lop3(p, stream);
     case BCNN_ENGINE_MMA_B1:
@@ -170,6 +174,17 @@ int bcnn_gemm_b1_engine(int engine, const void *A_bits, const void *W_bits, cons
     const int st = gemm_problem(p, A_bits, W_bits, thr, out, M, N, K, thr != nullptr);
     if (st != BCNN_OK) return st;
     return dispatch(engine, p, static_cast<cudaStream_t>(stream));
+}
+
+int bcnn_auto_engine(int B, int H, int W, int C_in, int C_out, int kh, int kw, int stride, int pad, int fused)
+{
+    ConvProblem p;
+    // validation only looks at pointer alignment and nullness: hand it aligned dummies
+    void *dummy = reinterpret_cast<void *>(uintptr_t(4096));
+    const int st = make_conv_problem(p, dummy, dummy, fused ? static_cast<const int32_t *>(dummy) : nullptr, dummy,
+                                     B, H, W, C_in, C_out, kh, kw, stride, pad, fused != 0);
+    if (st != BCNN_OK) return st;
+    return auto_engine(p);
 }
 
 int bcnn_device_error(void)

@@ -31,6 +31,15 @@ __device__ __forceinline__ void mma_u8(int (&d)[4], uint32_t a0, uint32_t a1, ui
         : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b.x), "r"(b.y));
 }
 
+// Output-channel permutation.  Inside each group of 32 output channels, column c (0..7) of
+// MMA atom j (0..3) carries channel 8*(c >> 1) + 2*j + (c & 1).  Thread q of a quad holds
+// columns 2q, 2q+1 of every atom, i.e. the eight consecutive channels 8q .. 8q+7: one byte
+// of the packed output word, or two 16-byte int32 stores.
+__device__ __forceinline__ int atom_col_to_channel(int atom, int c)
+{
+    return 32 * (atom >> 2) + 8 * (c >> 1) + 2 * (atom & 3) + (c & 1);
+}
+
 template <int NA, bool FUSED>
 __global__ void __launch_bounds__(THREADS, 2)
 conv_mma_s8_kernel(const ConvProblem p)
@@ -38,16 +47,18 @@ conv_mma_s8_kernel(const ConvProblem p)
     constexpr int BN = 8 * NA;
     extern __shared__ __align__(16) unsigned char smem[];
     uint2 *wfrag = reinterpret_cast<uint2 *>(smem);                 // [kwords][NA][32 lanes]
-    int *colc = reinterpret_cast<int *>(wfrag + (size_t)p.kwords * NA * 32);   // [BN] per-column constant
+    int *colc = reinterpret_cast<int *>(wfrag + (size_t)p.kwords * NA * 32);   // [BN] per-channel constant
+    int *tapoff = colc + BN;                                         // [kh*kw] word offset of each tap
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int g = lane >> 2, q = lane & 3;
     const int n0 = blockIdx.y * BN;
+    const int ntaps = p.kh * p.kw;
 
-    // ---- weight fragments in fragment order + per-column constants
+    // ---- weight fragments in fragment order, per-channel constants, tap offsets
     for (int idx = tid; idx < p.kwords * NA * 32; idx += THREADS) {
         const int l = idx & 31, j = (idx >> 5) % NA, kw = idx / (32 * NA);
-        const int n = n0 + 8 * j + (l >> 2), ql = l & 3;
+        const int n = n0 + atom_col_to_channel(j, l >> 2), ql = l & 3;
         const uint32_t w = (n < p.C_out) ? __ldg(p.w + (long)n * p.kwords + kw) : 0u;
         uint2 f;
         f.x = ((w >> ql) & 0x01010101u) << (7 - ql);
@@ -59,18 +70,20 @@ conv_mma_s8_kernel(const ConvProblem p)
         int pop = 0;
         if (n < p.C_out)
             for (int kw = 0; kw < p.kwords; ++kw) pop += __popc(__ldg(p.w + (long)n * p.kwords + kw));
-        // int32 output: value = colc - 2*pa + (acc >> 5);  fused: bit = (acc >> 5) - 2*pa >= thr - colc
-        const int base = p.K - 2 * pop;
-        colc[c] = FUSED ? ((n < p.C_out ? __ldg(p.thr + n) : 0) - base) : base;
+        // with acc = 128 * popc(A and G) and pa = popc(A):
+        //   int32:  value = (acc >> 5) - 2*pa + (K - 2*pop)
+        //   fused:  bit   = acc - 64*pa - 32*(thr - K + 2*pop) >= 0
+        colc[c] = FUSED ? -32 * ((n < p.C_out ? __ldg(p.thr + n) : 0) - p.K + 2 * pop) : p.K - 2 * pop;
     }
+    for (int tp = tid; tp < ntaps; tp += THREADS) tapoff[tp] = ((tp / p.kw) * p.W + (tp % p.kw)) * p.cw;
     __syncthreads();
 
-    // per-thread column constants: columns 8j + 2q + e
+    // per-thread channel constants: atom j, column 2q+e -> channel 32*(j/4) + 8q + 2*(j%4) + e
     int cc[NA][2];
 #pragma unroll
     for (int j = 0; j < NA; ++j) {
-        cc[j][0] = colc[8 * j + 2 * q];
-        cc[j][1] = colc[8 * j + 2 * q + 1];
+        cc[j][0] = colc[atom_col_to_channel(j, 2 * q)];
+        cc[j][1] = colc[atom_col_to_channel(j, 2 * q + 1)];
     }
 
     const uint32_t mlo = 0x01010101u << q, mhi = 0x10101010u << q;
@@ -78,24 +91,60 @@ conv_mma_s8_kernel(const ConvProblem p)
     const long nblocks = ((long)p.M + rows_per_iter - 1) / rows_per_iter;
     const long wstride = (long)gridDim.x * (THREADS / 32);
     const int owords = p.C_out >> 5;
+    const bool plain = (ntaps == 1 && p.stride == 1 && p.pad == 0);   // 1x1: row m is pixel m
 
-    for (long blk = (long)blockIdx.x * (THREADS / 32) + warp; blk < nblocks; blk += wstride) {
+    // Row set-up of one 32-row block: pointer to each window's top-left pixel (may lie outside the
+    // image) and one validity bit per tap.  Rows of this thread: mbase + 16*a + g + 8*h.
+    auto setup_rows = [&](long blk, const uint32_t *(&xb)[MA][2], uint32_t (&vmask)[MA][2]) {
         const int mbase = (int)(blk * rows_per_iter);
-        // rows handled by this thread: mbase + 16*a + g + 8*h
-        const uint32_t *xb[MA][2];
-        int ih0[MA][2], iw0[MA][2];
-        bool ok[MA][2];
 #pragma unroll
         for (int a = 0; a < MA; ++a)
 #pragma unroll
             for (int h = 0; h < 2; ++h) {
                 const int m = mbase + 16 * a + g + 8 * h;
-                ok[a][h] = m < p.M;
-                const RowCoord rc = row_coord(p, ok[a][h] ? m : 0);
-                xb[a][h] = p.x + (long)rc.b * p.H * p.W * p.cw;
-                ih0[a][h] = rc.ih0;
-                iw0[a][h] = rc.iw0;
+                const bool ok = m < p.M;
+                if (plain) {
+                    xb[a][h] = p.x + (long)(ok ? m : 0) * p.cw;
+                    vmask[a][h] = ok ? 1u : 0u;
+                } else {
+                    const RowCoord rc = row_coord(p, ok ? m : 0);
+                    xb[a][h] = p.x + (((long)rc.b * p.H + rc.ih0) * p.W + rc.iw0) * p.cw;
+                    uint32_t colbits = 0, mask = 0;
+                    for (int t = 0; t < p.kw; ++t)
+                        if (rc.iw0 + t >= 0 && rc.iw0 + t < p.W) colbits |= 1u << t;
+                    for (int r = 0; r < p.kh; ++r)
+                        if (rc.ih0 + r >= 0 && rc.ih0 + r < p.H) mask |= colbits << (r * p.kw);
+                    vmask[a][h] = ok ? mask : 0u;
+                }
             }
+    };
+    auto load_words = [&](uint32_t (&w)[MA][2], const uint32_t *const (&xb)[MA][2], const uint32_t (&vmask)[MA][2],
+                          int tap, int cj) {
+        const int off = tapoff[tap] + cj;
+#pragma unroll
+        for (int a = 0; a < MA; ++a)
+#pragma unroll
+            for (int h = 0; h < 2; ++h)
+                w[a][h] = ((vmask[a][h] >> tap) & 1u) ? __ldg(xb[a][h] + off) : 0u;
+    };
+
+    long blk = (long)blockIdx.x * (THREADS / 32) + warp;
+    const uint32_t *xb[MA][2];
+    uint32_t vmask[MA][2];
+    uint32_t w[MA][2];
+    if (blk < nblocks) {
+        setup_rows(blk, xb, vmask);
+        load_words(w, xb, vmask, 0, 0);
+    }
+    for (; blk < nblocks; blk += wstride) {
+        const int mbase = (int)(blk * rows_per_iter);
+        // the next block's rows are set up now so that its first words can be requested
+        // before this block's epilogue (the whole flattened K sequence is software-pipelined)
+        const long nblk = blk + wstride;
+        const uint32_t *xbn[MA][2];
+        uint32_t vmaskn[MA][2];
+        if (nblk < nblocks) setup_rows(nblk, xbn, vmaskn);
+
         int acc[MA][NA][4];
         int pa[MA][2];
 #pragma unroll
@@ -107,28 +156,12 @@ conv_mma_s8_kernel(const ConvProblem p)
                 for (int e = 0; e < 4; ++e) acc[a][j][e] = 0;
         }
 
-        // K loop, software-pipelined: the words of step kw+1 are in flight while step kw is multiplied
-        int r = 0, t = 0, cj = 0;      // tap and channel word of the K word being loaded (warp-uniform)
-        auto load_words = [&](uint32_t (&w)[MA][2]) {
-#pragma unroll
-            for (int a = 0; a < MA; ++a)
-#pragma unroll
-                for (int h = 0; h < 2; ++h) {
-                    const int ih = ih0[a][h] + r, iw = iw0[a][h] + t;
-                    uint32_t v = 0;
-                    if (ok[a][h] && ih >= 0 && ih < p.H && iw >= 0 && iw < p.W)
-                        v = __ldg(xb[a][h] + ((long)ih * p.W + iw) * p.cw + cj);
-                    w[a][h] = v;
-                }
-            if (++cj == p.cw) {
-                cj = 0;
-                if (++t == p.kw) { t = 0; ++r; }
-            }
-        };
-        uint32_t w[MA][2], wn[MA][2];
-        load_words(w);
+        int tap = 0, cj = 0;           // tap and channel word of the K word being loaded (warp-uniform)
         for (int kw = 0; kw < p.kwords; ++kw) {
-            if (kw + 1 < p.kwords) load_words(wn);
+            uint32_t wn[MA][2];
+            if (++cj == p.cw) { cj = 0; ++tap; }
+            if (kw + 1 < p.kwords) load_words(wn, xb, vmask, tap, cj);
+            else if (nblk < nblocks) load_words(wn, xbn, vmaskn, 0, 0);
             const uint2 *wf = wfrag + (size_t)kw * NA * 32 + lane;
 #pragma unroll
             for (int a = 0; a < MA; ++a) {
@@ -148,45 +181,58 @@ conv_mma_s8_kernel(const ConvProblem p)
                 w[a][1] = wn[a][1];
             }
         }
+#pragma unroll
+        for (int a = 0; a < MA; ++a)
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+                xb[a][h] = xbn[a][h];
+                vmask[a][h] = vmaskn[a][h];
+            }
 
-        // ---- epilogue.  acc[a][j][0,1] -> row g, columns 8j+2q, 8j+2q+1;  [2,3] -> row g+8.
+        // ---- epilogue.  acc[a][j][0,1] -> row g, columns 2q, 2q+1 of atom j;  [2,3] -> row g+8.
 #pragma unroll
         for (int a = 0; a < MA; ++a)
 #pragma unroll
             for (int h = 0; h < 2; ++h) {
                 const int m = mbase + 16 * a + g + 8 * h;
-                const int pa2 = 2 * pa[a][h];
                 if (!FUSED) {
+                    const int rowc = -2 * pa[a][h];
                     if (m < p.M) {
-                        int32_t *dst = static_cast<int32_t *>(p.out) + (long)m * p.C_out + n0 + 2 * q;
 #pragma unroll
-                        for (int j = 0; j < NA; ++j) {
-                            const int n = n0 + 8 * j + 2 * q;
-                            const int v0 = cc[j][0] - pa2 + (acc[a][j][2 * h] >> 5);
-                            const int v1 = cc[j][1] - pa2 + (acc[a][j][2 * h + 1] >> 5);
-                            if (n + 1 < p.C_out && (p.C_out & 1) == 0) {
-                                *reinterpret_cast<int2 *>(dst + 8 * j) = make_int2(v0, v1);
+                        for (int gi = 0; gi < NA / 4; ++gi) {
+                            const int n = n0 + 32 * gi + 8 * q;      // this thread's 8 consecutive channels
+                            int v[8];
+#pragma unroll
+                            for (int jj = 0; jj < 4; ++jj)
+#pragma unroll
+                                for (int e = 0; e < 2; ++e)
+                                    v[2 * jj + e] = (acc[a][4 * gi + jj][2 * h + e] >> 5) + rowc + cc[4 * gi + jj][e];
+                            int32_t *dst = static_cast<int32_t *>(p.out) + (long)m * p.C_out + n;
+                            if ((p.C_out & 3) == 0 && n + 8 <= p.C_out) {
+                                *reinterpret_cast<int4 *>(dst) = make_int4(v[0], v[1], v[2], v[3]);
+                                *reinterpret_cast<int4 *>(dst + 4) = make_int4(v[4], v[5], v[6], v[7]);
                             } else {
-                                if (n < p.C_out) dst[8 * j] = v0;
-                                if (n + 1 < p.C_out) dst[8 * j + 1] = v1;
+#pragma unroll
+                                for (int i = 0; i < 8; ++i)
+                                    if (n + i < p.C_out) dst[i] = v[i];
                             }
                         }
                     }
                 } else {
+                    const int rowc = -64 * pa[a][h];
 #pragma unroll
-                    for (int wd = 0; wd < NA / 4; ++wd) {
-                        uint32_t bits = 0;
+                    for (int gi = 0; gi < NA / 4; ++gi) {
+                        // shift the sign bits of (acc + rowc + colc) in, highest channel first
+                        uint32_t sb = 0;
 #pragma unroll
-                        for (int jj = 0; jj < 4; ++jj) {
-                            const int j = 4 * wd + jj;
-                            const int v0 = (acc[a][j][2 * h] >> 5) - pa2;
-                            const int v1 = (acc[a][j][2 * h + 1] >> 5) - pa2;
-                            bits |= (v0 >= cc[j][0] ? 1u : 0u) << (8 * jj + 2 * q);
-                            bits |= (v1 >= cc[j][1] ? 1u : 0u) << (8 * jj + 2 * q + 1);
-                        }
+                        for (int jj = 3; jj >= 0; --jj)
+#pragma unroll
+                            for (int e = 1; e >= 0; --e)
+                                sb = __funnelshift_l((uint32_t)(acc[a][4 * gi + jj][2 * h + e] + rowc + cc[4 * gi + jj][e]), sb, 1);
+                        uint32_t bits = (~sb & 0xffu) << (8 * q);
                         bits |= __shfl_xor_sync(0xffffffffu, bits, 1);
                         bits |= __shfl_xor_sync(0xffffffffu, bits, 2);
-                        const int nword = (n0 >> 5) + wd;
+                        const int nword = (n0 >> 5) + gi;
                         if (q == 0 && m < p.M && nword < owords)
                             static_cast<uint32_t *>(p.out)[(long)m * owords + nword] = bits;
                     }
@@ -195,7 +241,10 @@ conv_mma_s8_kernel(const ConvProblem p)
     }
 }
 
-size_t smem_bytes(const ConvProblem &p, int NA) { return (size_t)p.kwords * NA * 32 * sizeof(uint2) + 8 * NA * sizeof(int); }
+size_t smem_bytes(const ConvProblem &p, int NA)
+{
+    return (size_t)p.kwords * NA * 32 * sizeof(uint2) + 8 * NA * sizeof(int) + (size_t)p.kh * p.kw * sizeof(int);
+}
 
 template <int NA>
 int launch_na(const ConvProblem &p, cudaStream_t stream)
@@ -228,6 +277,7 @@ bool conv_mma_s8_supports(const ConvProblem &p)
 {
     if (p.thr != nullptr && (p.C_out % 32 != 0)) return false;
     const int NA = p.C_out <= 32 ? 4 : 8;
+    if (p.kh * p.kw > 32) return false;     // one validity bit per tap in a 32-bit mask
     return smem_bytes(p, NA) <= (size_t)MAX_SMEM && p.K <= (1 << 20);
 }
 
