@@ -304,7 +304,8 @@ def run_gpu(args):
     tensor_peak = 2.0 * peaks["bf16_tflops_sustained"]
     engines = [binding.bcnn_auto_engine(B, l.H, l.W, l.C_in, l.C_out, l.k, l.k, l.stride, l.pad) for l in layers]
     kernel_of = {"tc_i8": "conv_tc_i8_kernel (tcgen05 kind::i8)", "mma_s8": "conv_mma_s8_kernel (mma.sync u8)",
-                 "mma_b1": "conv_mma_b1_kernel (mma.sync b1)", "lop3": "conv_lop3_kernel (xor + popc)"}
+                 "mma_b1": "conv_mma_b1_kernel (mma.sync b1)",
+                 "tc_ws": "conv_tc_ws_kernel (tcgen05 kind::i8, weights resident in shared memory)", "lop3": "conv_lop3_kernel (xor + popc)"}
     per_layer = [{"layer": l.name, "engine": engines[i], "ms": float(per_ms[i + 1]),
                   "tops": l.ops(B) / (per_ms[i + 1] / 1e3) / 1e12} for i, l in enumerate(layers)]
     groups = []
@@ -458,7 +459,7 @@ def run_sweep(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--mode", default="bench", choices=["bench", "sweep"])
-    ap.add_argument("--engines", default="auto,lop3,mma_b1,tc_i8,mma_s8")
+    ap.add_argument("--engines", default="auto,lop3,mma_b1,tc_i8,mma_s8,tc_ws")
     ap.add_argument("--sweep-set", default="all", choices=["gemm", "conv", "all"])
     ap.add_argument("--only", default="", help="sweep mode: run only shapes whose label contains this text")
     ap.add_argument("--outs", default="int32,fused", help="sweep mode: output kinds to run")

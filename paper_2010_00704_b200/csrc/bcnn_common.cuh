@@ -67,6 +67,8 @@ int launch_conv_mma_b1(const ConvProblem &p, cudaStream_t stream);
 bool conv_mma_b1_supports(const ConvProblem &p);
 int launch_conv_mma_s8(const ConvProblem &p, cudaStream_t stream);
 bool conv_mma_s8_supports(const ConvProblem &p);
+int launch_conv_tc_ws(const ConvProblem &p, cudaStream_t stream);
+bool conv_tc_ws_supports(const ConvProblem &p);
 int launch_conv_tc_i8(const ConvProblem &p, cudaStream_t stream);
 bool conv_tc_i8_supports(const ConvProblem &p);
 int *device_error_word();   // device address of the error word of the current device (nullptr on failure)

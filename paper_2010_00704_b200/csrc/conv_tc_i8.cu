@@ -36,7 +36,10 @@ constexpr int BM = 128;
 constexpr int ROWB = 128;                 // bytes of one expanded tile row per stage (= 128 bits of K)
 constexpr int EPI_WARPS = 4;
 constexpr int FIRST_PRODUCER_THREAD = 32 * (1 + EPI_WARPS);
-constexpr uint32_t WAIT_LIMIT = 1u << 22; // polls before a wait gives up
+constexpr uint32_t WAIT_LIMIT = 1u << 22;
+// upper bound (ns) for which one try_wait may suspend the thread: waiting warps then leave
+// the issue slots to the warps that have work; the wake-up on phase completion is immediate
+constexpr uint32_t SUSPEND_HINT_NS = 20000; // polls before a wait gives up
 
 constexpr int ERR_PRODUCER_TIMEOUT = 101;
 constexpr int ERR_MMA_TIMEOUT = 102;
@@ -77,9 +80,9 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
     uint32_t ok;
     asm volatile(
         "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
         "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+        : "=r"(ok) : "r"(bar), "r"(parity), "r"(SUSPEND_HINT_NS) : "memory");
     return ok != 0;
 }
 
@@ -115,18 +118,20 @@ __device__ __forceinline__ void tc_mma_i8(uint32_t d_tmem, uint64_t a_desc, uint
         : "memory");
 }
 
+// 32 accumulator columns of this warp's 32 rows.  The load and its completion wait are one asm
+// statement so that no use of the destination registers can be scheduled between them.
 __device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&v)[32])
 {
     asm volatile(
         "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
         "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
-        "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+        "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];\n\t"
+        "tcgen05.wait::ld.sync.aligned;"
         : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
           "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
           "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
           "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
-        : "r"(taddr));
-    asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+        : "r"(taddr) : "memory");
 }
 
 // Shared-memory matrix descriptor of a K-major tile with 128-byte rows and the 128-byte

@@ -17,7 +17,7 @@ def bk():
     return binding
 
 
-ENGINES = ["auto", "lop3", "mma_b1", "tc_i8", "mma_s8"]
+ENGINES = ["auto", "lop3", "mma_b1", "tc_i8", "mma_s8", "tc_ws"]
 
 
 def dev(a):
