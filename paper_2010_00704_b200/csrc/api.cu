@@ -76,7 +76,7 @@ int make_conv_problem(ConvProblem &p, const void *x, const void *w, const int32_
 //   * the single-bit mma.sync and CUDA-core engines never win and serve as fallbacks.
 int auto_engine(const ConvProblem &p)
 {
-    if (p.C_out <= 128 && p.C_out >= 64 && p.K >= 256 && conv_tc_ws_supports(p)) return BCNN_ENGINE_TC_WS;
+    if (p.C_out <= 128 && p.C_out >= 64 && p.K >= 256 - 128 * (p.C_out > 64) && conv_tc_ws_supports(p)) return BCNN_ENGINE_TC_WS;
     if (p.C_out <= 64 && conv_mma_s8_supports(p)) return BCNN_ENGINE_MMA_S8;
     if (conv_tc_i8_supports(p)) return BCNN_ENGINE_TC_I8;
     if (conv_mma_b1_supports(p)) return BCNN_ENGINE_MMA_B1;

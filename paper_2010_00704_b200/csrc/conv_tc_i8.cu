@@ -36,10 +36,10 @@ constexpr int BM = 128;
 constexpr int ROWB = 128;                 // bytes of one expanded tile row per stage (= 128 bits of K)
 constexpr int EPI_WARPS = 4;
 constexpr int FIRST_PRODUCER_THREAD = 32 * (1 + EPI_WARPS);
-constexpr uint32_t WAIT_LIMIT = 1u << 22;
+constexpr uint32_t WAIT_LIMIT = 1u << 17;
 // upper bound (ns) for which one try_wait may suspend the thread: waiting warps then leave
 // the issue slots to the warps that have work; the wake-up on phase completion is immediate
-constexpr uint32_t SUSPEND_HINT_NS = 20000; // polls before a wait gives up
+constexpr uint32_t SUSPEND_HINT_NS = 20000;
 
 constexpr int ERR_PRODUCER_TIMEOUT = 101;
 constexpr int ERR_MMA_TIMEOUT = 102;

@@ -30,7 +30,7 @@ constexpr int EPI_WARPS = 4;
 constexpr int FIRST_PRODUCER_THREAD = 32 * (1 + EPI_WARPS);
 constexpr int PF = 3;                     // packed-word stages in flight per producer thread
 constexpr int MAX_SMEM = 227 * 1024;
-constexpr uint32_t WAIT_LIMIT = 1u << 22;
+constexpr uint32_t WAIT_LIMIT = 1u << 17;
 // upper bound (ns) for which one try_wait may suspend the thread: waiting warps then leave
 // the issue slots to the warps that have work; the wake-up on phase completion is immediate
 constexpr uint32_t SUSPEND_HINT_NS = 20000;
@@ -307,9 +307,10 @@ conv_tc_ws_kernel(const ConvProblem p)
                     tc_fence_after();
                     const uint64_t a_desc = make_desc(ring + (uint32_t)s * C::A_BYTES);
                     const uint64_t b_desc = make_desc(wexp + (uint32_t)kt * C::W_TILE_BYTES);
+                    const int nk = p.kwords - 4 * kt;             // 32 bits of K per instruction; skip the zero tail
 #pragma unroll
                     for (int k = 0; k < 4; ++k)
-                        tc_mma_i8(d_tmem, a_desc + 2u * k, b_desc + 2u * k, idesc, (kt > 0 || k > 0) ? 1u : 0u);
+                        if (k < nk) tc_mma_i8(d_tmem, a_desc + 2u * k, b_desc + 2u * k, idesc, (kt > 0 || k > 0) ? 1u : 0u);
                     tc_commit(empty_bar(s));
                     if (++s == STAGES) { s = 0; ring_phase ^= 1u; }
                 }
@@ -515,8 +516,10 @@ int launch_ws(const ConvProblem &p0, cudaStream_t stream)
     return cudaGetLastError() == cudaSuccess ? BCNN_OK : BCNN_ERR_CUDA;
 }
 
+// Parity waits are only safe while a waiter is at most one phase behind.  A producer group comes back
+// to the ring every G stages and completion is in order, so the ring must hold at least G stages.
 template <int BN, int G>
-bool fits(const ConvProblem &p) { return ws_layout<BN, G>(p.kwords).a_stages >= 3; }
+bool fits(const ConvProblem &p) { return ws_layout<BN, G>(p.kwords).a_stages >= G; }
 
 }  // namespace
 
@@ -528,7 +531,7 @@ bool conv_tc_ws_supports(const ConvProblem &p)
     if ((long)(p.kh * (long)p.W + p.kw) * p.cw >= (1L << 26)) return false;
     if (p.C_out <= 32) return fits<32, 4>(p);
     if (p.C_out <= 64) return fits<64, 4>(p);
-    return fits<128, 4>(p);
+    return fits<128, 4>(p) || fits<128, 2>(p);
 }
 
 int launch_conv_tc_ws(const ConvProblem &p, cudaStream_t stream)
@@ -536,7 +539,8 @@ int launch_conv_tc_ws(const ConvProblem &p, cudaStream_t stream)
     if (!conv_tc_ws_supports(p)) return BCNN_ERR_UNSUPPORTED;
     if (p.C_out <= 32) return launch_ws<32, 4>(p, stream);
     if (p.C_out <= 64) return launch_ws<64, 4>(p, stream);
-    return launch_ws<128, 4>(p, stream);
+    if (fits<128, 4>(p)) return launch_ws<128, 4>(p, stream);
+    return launch_ws<128, 2>(p, stream);     // long K: fewer producer groups leave room for the ring
 }
 
 }  // namespace bcnn
