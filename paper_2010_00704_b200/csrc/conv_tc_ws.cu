@@ -15,6 +15,8 @@
 //     are being gathered / expanded at any time (one thread's stage latency is several
 //     hundred cycles, an MMA stage as little as 64);
 //   * up to four accumulator buffers, so the epilogue of one tile overlaps the MMAs of the next ones;
+//   * the warp that issues the MMAs waits only on named barriers; a separate control warp does the
+//     mbarrier waits for it (a memory instruction after tensor-core instructions stalls the issuer);
 //   * the implicit-im2col gather uses a per-K-word table (tap, word offset) and a per-row
 //     tap-validity mask instead of divisions; out-of-image taps are zero-filled by cp.async.
 // Every mbarrier wait is bounded and reports through the device error word.
@@ -34,6 +36,7 @@ constexpr uint32_t WAIT_LIMIT = 1u << 17;
 // upper bound (ns) for which one try_wait may suspend the thread: waiting warps then leave
 // the issue slots to the warps that have work; the wake-up on phase completion is immediate
 constexpr uint32_t SUSPEND_HINT_NS = 20000;
+constexpr uint32_t SLEEP_NS = 100;
 
 constexpr int ERR_PRODUCER_TIMEOUT = 111;
 constexpr int ERR_MMA_TIMEOUT = 112;
@@ -42,7 +45,8 @@ constexpr int ERR_EPILOGUE_TIMEOUT = 113;
 template <int BN, int G> struct Cfg {
     static constexpr int BNX = BN + 16;                       // + the all-ones row (MMA N is a multiple of 16)
     static constexpr int PROD_THREADS = G * BM;
-    static constexpr int THREADS = FIRST_PRODUCER_THREAD + PROD_THREADS;
+    static constexpr int CONTROL_WARP = (FIRST_PRODUCER_THREAD + PROD_THREADS) / 32;   // last warp
+    static constexpr int THREADS = FIRST_PRODUCER_THREAD + PROD_THREADS + 32;
     static constexpr int NBUF = (BNX * 4 <= 512) ? 4 : 3;     // accumulator buffers in tensor memory
     static constexpr int TMEM_COLS = (NBUF * BNX <= 128) ? 128 : (NBUF * BNX <= 256 ? 256 : 512);
     static constexpr int A_BYTES = BM * ROWB;
@@ -70,9 +74,13 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
         : "=r"(ok) : "r"(bar), "r"(parity), "r"(SUSPEND_HINT_NS) : "memory");
     return ok != 0;
 }
+// Bounded wait with back-off.  A polling warp competes with the MMA-issuing warp for issue
+// slots, so after a first failed poll the waiter sleeps between polls.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *err, int code)
 {
+    if (mbar_try_wait(bar, parity)) return true;
     for (uint32_t it = 0; it < WAIT_LIMIT; ++it) {
+        __nanosleep(SLEEP_NS);
         if (mbar_try_wait(bar, parity)) return true;
         if ((it & 255u) == 255u && *abort_flag) return false;
     }
@@ -96,6 +104,30 @@ __device__ __forceinline__ void tc_mma_i8(uint32_t d_tmem, uint64_t a_desc, uint
         ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(0u), "r"(0u), "r"(0u), "r"(0u)
         : "memory");
 }
+// Predicated forms for the issuer warp: every lane executes the same straight-line code and
+// only the elected lane's predicate is true, so there is no branch to reconverge from.  The
+// descriptors are passed as (low word, high word); only the low word (start address) varies.
+__device__ __forceinline__ void tc_mma_i8_pred(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t desc_hi,
+                                               uint32_t idesc, uint32_t accumulate, uint32_t pred)
+{
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t.reg .b64 da, db;\n\t"
+        "setp.ne.b32 p, %5, 0;\n\t"
+        "setp.ne.b32 q, %6, 0;\n\t"
+        "mov.b64 da, {%1, %3};\n\t"
+        "mov.b64 db, {%2, %3};\n\t"
+        "@q tcgen05.mma.cta_group::1.kind::i8 [%0], da, db, %4, {%7, %7, %7, %7}, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(desc_hi), "r"(idesc), "r"(accumulate), "r"(pred), "r"(0u)
+        : "memory");
+}
+__device__ __forceinline__ void tc_commit_pred(uint32_t bar, uint32_t pred)
+{
+    asm volatile(
+        "{\n\t.reg .pred q;\n\tsetp.ne.b32 q, %1, 0;\n\t"
+        "@q tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n\t}"
+        ::"r"(bar), "r"(pred) : "memory");
+}
+
 // 32 accumulator columns of this warp's 32 rows.  The load and its completion wait are one asm
 // statement so that no use of the destination registers can be scheduled between them.
 __device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&v)[32])
@@ -289,36 +321,59 @@ conv_tc_ws_kernel(const ConvProblem p)
 
     if (warp == 0) {
         // ------------------------------------------------------------------ MMA issuer
-        if (lane == 0) {
-            constexpr uint32_t idesc = make_idesc(BNX);
-            int s = 0;
-            uint32_t ring_phase = 0;
-            bool alive = true;
-            int buf = 0;
-            uint32_t buf_phase = 1;          // first use of every buffer: free
-            for (int ti = 0; ti < my_tiles && alive; ++ti) {
-                alive = mbar_wait(tempty_bar(buf), buf_phase, abort_flag, p.err, ERR_MMA_TIMEOUT);
-                if (!alive) break;
+        // This warp never touches memory: a load or an mbarrier wait issued after tensor-core
+        // instructions holds the issuing thread until they have drained (measured: +230 cycles per
+        // stage), a named barrier does not.  The control warp does the waiting and releases one
+        // stage at a time through named barrier 1 + slot.
+        constexpr uint32_t idesc = make_idesc(BNX);
+        const uint64_t desc0 = make_desc(0);
+        const uint32_t desc_hi = (uint32_t)(desc0 >> 32);
+        const uint32_t a_lo0 = (uint32_t)desc0 | ((ring & 0x3FFFFu) >> 4);       // + slot * (A_BYTES / 16)
+        const uint32_t b_lo0 = (uint32_t)desc0 | ((wexp & 0x3FFFFu) >> 4);       // + kt * (W_TILE_BYTES / 16)
+        const uint32_t elected = lane == 0 ? 1u : 0u;
+        int s = 0, buf = 0;
+        for (int ti = 0; ti < my_tiles; ++ti) {
+            const uint32_t d_tmem = tmem_base + (uint32_t)(buf * BNX);
+            const uint32_t tfull = tfull_bar(buf);
+            for (int kt = 0; kt < ktiles; ++kt) {
+                const uint32_t a_lo = a_lo0 + (uint32_t)s * (C::A_BYTES >> 4);
+                const uint32_t b_lo = b_lo0 + (uint32_t)kt * (C::W_TILE_BYTES >> 4);
+                const int nk = p.kwords - 4 * kt;                 // 32 bits of K per instruction; skip the zero tail
+                const uint32_t e1 = nk > 1 ? elected : 0u, e2 = nk > 2 ? elected : 0u, e3 = nk > 3 ? elected : 0u;
+                const uint32_t last = (kt == ktiles - 1) ? elected : 0u;
+                const uint32_t ebar = empty_bar(s);
+                asm volatile("bar.sync %0, 64;" ::"r"(1 + s) : "memory");
                 tc_fence_after();
-                const uint32_t d_tmem = tmem_base + (uint32_t)(buf * BNX);
-                for (int kt = 0; kt < ktiles; ++kt) {
-                    alive = mbar_wait(full_bar(s), ring_phase, abort_flag, p.err, ERR_MMA_TIMEOUT);
-                    if (!alive) break;
-                    tc_fence_after();
-                    const uint64_t a_desc = make_desc(ring + (uint32_t)s * C::A_BYTES);
-                    const uint64_t b_desc = make_desc(wexp + (uint32_t)kt * C::W_TILE_BYTES);
-                    const int nk = p.kwords - 4 * kt;             // 32 bits of K per instruction; skip the zero tail
-#pragma unroll
-                    for (int k = 0; k < 4; ++k)
-                        if (k < nk) tc_mma_i8(d_tmem, a_desc + 2u * k, b_desc + 2u * k, idesc, (kt > 0 || k > 0) ? 1u : 0u);
-                    tc_commit(empty_bar(s));
-                    if (++s == STAGES) { s = 0; ring_phase ^= 1u; }
-                }
-                if (alive) tc_commit(tfull_bar(buf));
-                if (++buf == NBUF) { buf = 0; buf_phase ^= 1u; }
+                tc_mma_i8_pred(d_tmem, a_lo, b_lo, desc_hi, idesc, kt > 0 ? 1u : 0u, elected);   // +2 per 32 bytes of K
+                tc_mma_i8_pred(d_tmem, a_lo + 2u, b_lo + 2u, desc_hi, idesc, 1u, e1);
+                tc_mma_i8_pred(d_tmem, a_lo + 4u, b_lo + 4u, desc_hi, idesc, 1u, e2);
+                tc_mma_i8_pred(d_tmem, a_lo + 6u, b_lo + 6u, desc_hi, idesc, 1u, e3);
+                tc_commit_pred(ebar, elected);
+                tc_commit_pred(tfull, last);
+                if (++s == STAGES) s = 0;
             }
+            if (++buf == NBUF) buf = 0;
         }
-        __syncwarp();
+    } else if (warp == C::CONTROL_WARP) {
+        // ------------------------------------------------------------------ control: waits for the issuer
+        // Stage `it` is released (bar.arrive on 1 + slot) once its ring slot is full and, for a tile's
+        // first stage, once the accumulator buffer is free.  The slot being full implies that the
+        // issuer is past the previous use of the same named barrier (it committed that slot's release).
+        // After a time-out the remaining stages are released without waiting so that the issuer,
+        // whose barrier wait has no time limit, always terminates; the error word tells the host.
+        int s = 0, buf = 0;
+        uint32_t ring_phase = 0, buf_phase = 1;      // first use of every accumulator buffer: free
+        bool alive = true;
+        for (int ti = 0; ti < my_tiles; ++ti) {
+            if (lane == 0 && alive) alive = mbar_wait(tempty_bar(buf), buf_phase, abort_flag, p.err, ERR_MMA_TIMEOUT);
+            for (int kt = 0; kt < ktiles; ++kt) {
+                if (lane == 0 && alive) alive = mbar_wait(full_bar(s), ring_phase, abort_flag, p.err, ERR_MMA_TIMEOUT);
+                __syncwarp();
+                asm volatile("bar.arrive %0, 64;" ::"r"(1 + s) : "memory");
+                if (++s == STAGES) { s = 0; ring_phase ^= 1u; }
+            }
+            if (++buf == NBUF) { buf = 0; buf_phase ^= 1u; }
+        }
     } else if (warp <= EPI_WARPS) {
         // ------------------------------------------------------------------ epilogue
         const int quad = warp & 3;
