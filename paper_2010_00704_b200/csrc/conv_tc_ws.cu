@@ -8,6 +8,10 @@
 // Differences, all aimed at short tiles (a 128 x 32 x 32 tile is one MMA instruction):
 //   * the CTA expands its weight tile ONCE into shared memory and keeps it for all its
 //     output tiles; only activations stream through the ring;
+//   * the activation ring lives in TENSOR memory, not shared memory: producers write expanded rows
+//     with tcgen05.st and the MMA takes its A operand from tensor memory.  A narrow MMA is bound by
+//     operand fetch from shared memory (128 x 32 bytes of A per instruction whatever N is); with A in
+//     tensor memory only the small weight slice is fetched;
 //   * one extra all-ones weight row is appended, so column BN of every accumulator holds
 //     128 * popc(A) for its row: the epilogue reads the row popcount from tensor memory and
 //     no per-tile constants travel through shared memory;
@@ -47,9 +51,14 @@ template <int BN, int G> struct Cfg {
     static constexpr int PROD_THREADS = G * BM;
     static constexpr int CONTROL_WARP = (FIRST_PRODUCER_THREAD + PROD_THREADS) / 32;   // last warp
     static constexpr int THREADS = FIRST_PRODUCER_THREAD + PROD_THREADS + 32;
-    static constexpr int NBUF = (BNX * 4 <= 512) ? 4 : 3;     // accumulator buffers in tensor memory
-    static constexpr int TMEM_COLS = (NBUF * BNX <= 128) ? 128 : (NBUF * BNX <= 256 ? 256 : 512);
-    static constexpr int A_BYTES = BM * ROWB;
+    // Tensor memory (512 columns): NBUF accumulator buffers of BNX columns, then the activation ring,
+    // one stage = 128 rows x 128 expanded bytes = 32 columns.
+    static constexpr int NBUF = BN == 32 ? 4 : (BN == 64 ? 3 : 2);
+    static constexpr int STAGES = BN == 128 ? 7 : 8;
+    static constexpr int A_COL0 = NBUF * BNX;
+    static constexpr int TMEM_COLS = 512;
+    static_assert(A_COL0 + STAGES * 32 <= 512, "tensor memory budget");
+    static_assert(STAGES >= G, "a producer group must not lap the ring (parity waits)");
     static constexpr int W_TILE_BYTES = BNX * ROWB;           // one K stage of the expanded weights
     static constexpr int BITS_BYTES = PF * PROD_THREADS * 16;
 };
@@ -118,6 +127,34 @@ __device__ __forceinline__ void tc_mma_i8_pred(uint32_t d_tmem, uint32_t a_lo, u
         "mov.b64 db, {%2, %3};\n\t"
         "@q tcgen05.mma.cta_group::1.kind::i8 [%0], da, db, %4, {%7, %7, %7, %7}, p;\n\t}"
         ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(desc_hi), "r"(idesc), "r"(accumulate), "r"(pred), "r"(0u)
+        : "memory");
+}
+// A operand from tensor memory (128 lanes x 8 columns = 128 rows x 32 bytes of K), B from shared memory.
+__device__ __forceinline__ void tc_mma_i8_ts_pred(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t desc_hi,
+                                                  uint32_t idesc, uint32_t accumulate, uint32_t pred)
+{
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t.reg .b64 db;\n\t"
+        "setp.ne.b32 p, %5, 0;\n\t"
+        "setp.ne.b32 q, %6, 0;\n\t"
+        "mov.b64 db, {%2, %3};\n\t"
+        "@q tcgen05.mma.cta_group::1.kind::i8 [%0], [%1], db, %4, {%7, %7, %7, %7}, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_tmem), "r"(b_lo), "r"(desc_hi), "r"(idesc), "r"(accumulate), "r"(pred), "r"(0u)
+        : "memory");
+}
+// 32 columns of this warp's 32 lanes <- 32 registers; returns once the store has completed.
+__device__ __forceinline__ void tc_st32(uint32_t taddr, const uint32_t (&v)[32])
+{
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+        "{%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,"
+        "%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32};\n\t"
+        "tcgen05.wait::st.sync.aligned;"
+        ::"r"(taddr),
+          "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]),
+          "r"(v[8]), "r"(v[9]), "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15]),
+          "r"(v[16]), "r"(v[17]), "r"(v[18]), "r"(v[19]), "r"(v[20]), "r"(v[21]), "r"(v[22]), "r"(v[23]),
+          "r"(v[24]), "r"(v[25]), "r"(v[26]), "r"(v[27]), "r"(v[28]), "r"(v[29]), "r"(v[30]), "r"(v[31])
         : "memory");
 }
 __device__ __forceinline__ void tc_commit_pred(uint32_t bar, uint32_t pred)
@@ -203,7 +240,6 @@ __device__ __forceinline__ void expand_store_w(uint32_t w, uint32_t row_addr, in
 }
 
 struct WsLayout {
-    int a_stages;     // ring depth
     int ktiles;       // 128-bit K stages
     int smem;         // dynamic shared memory in bytes
 };
@@ -214,11 +250,10 @@ __host__ __device__ inline WsLayout ws_layout(int kwords)
     using C = Cfg<BN, G>;
     WsLayout l;
     l.ktiles = (kwords + 3) >> 2;
-    const int fixed = 1024 + l.ktiles * C::W_TILE_BYTES + C::BITS_BYTES + BN * 4 + l.ktiles * 4 * 4;
-    int st = (MAX_SMEM - 256 - fixed) / C::A_BYTES;
-    if (st > 8) st = 8;
-    l.a_stages = st;
-    l.smem = fixed + (st > 0 ? st : 0) * C::A_BYTES;
+    l.smem = 1024 + l.ktiles * C::W_TILE_BYTES + C::BITS_BYTES + BN * 4 + l.ktiles * 4 * 4;
+    // each CTA takes all 512 tensor-memory columns: ask for more than half of an SM's shared memory
+    // so that two CTAs of this kernel never share an SM (the second would sit in tcgen05.alloc)
+    if (l.smem < 120 * 1024) l.smem = 120 * 1024;
     return l;
 }
 
@@ -240,15 +275,14 @@ conv_tc_ws_kernel(const ConvProblem p)
     const int warp = tid >> 5, lane = tid & 31;
     const WsLayout L = ws_layout<BN, G>(p.kwords);
     const int ktiles = L.ktiles;
-    const int STAGES = L.a_stages;
+    constexpr int STAGES = C::STAGES;
     const int m_tiles = (p.M + BM - 1) / BM;
     const int my_tiles = ((int)blockIdx.x < m_tiles) ? (m_tiles - 1 - (int)blockIdx.x) / (int)gridDim.x + 1 : 0;
     const int total_items = my_tiles * ktiles;
 
     // shared-memory map (all 1024-byte aligned where the MMA reads)
     const uint32_t wexp = (smem_u32(smem_raw) + 1023u) & ~1023u;          // [ktiles][BNX rows][128 B]
-    const uint32_t ring = wexp + (uint32_t)ktiles * C::W_TILE_BYTES;      // [STAGES][128 rows][128 B]
-    const uint32_t bits_ring = ring + (uint32_t)STAGES * C::A_BYTES;      // [PF][PROD_THREADS][16 B]
+    const uint32_t bits_ring = wexp + (uint32_t)ktiles * C::W_TILE_BYTES; // [PF][PROD_THREADS][16 B]
     const uint32_t colc_addr = bits_ring + C::BITS_BYTES;                 // [BN] int32
     const uint32_t ktab_addr = colc_addr + BN * 4;                        // [ktiles*4] int32: (word offset << 5) | tap
     const uint32_t bar0 = smem_u32(bars);
@@ -328,7 +362,7 @@ conv_tc_ws_kernel(const ConvProblem p)
         constexpr uint32_t idesc = make_idesc(BNX);
         const uint64_t desc0 = make_desc(0);
         const uint32_t desc_hi = (uint32_t)(desc0 >> 32);
-        const uint32_t a_lo0 = (uint32_t)desc0 | ((ring & 0x3FFFFu) >> 4);       // + slot * (A_BYTES / 16)
+        const uint32_t a_tmem0 = tmem_base + (uint32_t)C::A_COL0;                // + slot * 32 columns
         const uint32_t b_lo0 = (uint32_t)desc0 | ((wexp & 0x3FFFFu) >> 4);       // + kt * (W_TILE_BYTES / 16)
         const uint32_t elected = lane == 0 ? 1u : 0u;
         int s = 0, buf = 0;
@@ -336,7 +370,7 @@ conv_tc_ws_kernel(const ConvProblem p)
             const uint32_t d_tmem = tmem_base + (uint32_t)(buf * BNX);
             const uint32_t tfull = tfull_bar(buf);
             for (int kt = 0; kt < ktiles; ++kt) {
-                const uint32_t a_lo = a_lo0 + (uint32_t)s * (C::A_BYTES >> 4);
+                const uint32_t a_t = a_tmem0 + (uint32_t)s * 32u;
                 const uint32_t b_lo = b_lo0 + (uint32_t)kt * (C::W_TILE_BYTES >> 4);
                 const int nk = p.kwords - 4 * kt;                 // 32 bits of K per instruction; skip the zero tail
                 const uint32_t e1 = nk > 1 ? elected : 0u, e2 = nk > 2 ? elected : 0u, e3 = nk > 3 ? elected : 0u;
@@ -344,10 +378,11 @@ conv_tc_ws_kernel(const ConvProblem p)
                 const uint32_t ebar = empty_bar(s);
                 asm volatile("bar.sync %0, 64;" ::"r"(1 + s) : "memory");
                 tc_fence_after();
-                tc_mma_i8_pred(d_tmem, a_lo, b_lo, desc_hi, idesc, kt > 0 ? 1u : 0u, elected);   // +2 per 32 bytes of K
-                tc_mma_i8_pred(d_tmem, a_lo + 2u, b_lo + 2u, desc_hi, idesc, 1u, e1);
-                tc_mma_i8_pred(d_tmem, a_lo + 4u, b_lo + 4u, desc_hi, idesc, 1u, e2);
-                tc_mma_i8_pred(d_tmem, a_lo + 6u, b_lo + 6u, desc_hi, idesc, 1u, e3);
+                // per 32 bytes of K: 8 tensor-memory columns of A, +2 (16-byte units) in the B descriptor
+                tc_mma_i8_ts_pred(d_tmem, a_t, b_lo, desc_hi, idesc, kt > 0 ? 1u : 0u, elected);
+                tc_mma_i8_ts_pred(d_tmem, a_t + 8u, b_lo + 2u, desc_hi, idesc, 1u, e1);
+                tc_mma_i8_ts_pred(d_tmem, a_t + 16u, b_lo + 4u, desc_hi, idesc, 1u, e2);
+                tc_mma_i8_ts_pred(d_tmem, a_t + 24u, b_lo + 6u, desc_hi, idesc, 1u, e3);
                 tc_commit_pred(ebar, elected);
                 tc_commit_pred(tfull, last);
                 if (++s == STAGES) s = 0;
@@ -456,8 +491,9 @@ conv_tc_ws_kernel(const ConvProblem p)
     } else {
         // ------------------------------------------------------------------ producers
         const int ptid = tid - FIRST_PRODUCER_THREAD;
-        const int grp = ptid >> 7, row = ptid & 127;             // group = 4 consecutive warps
-        const int xr = row & 7;
+        const int grp = ptid >> 7;                               // group = 4 consecutive warps
+        const int quad = warp & 3;                               // tensor-memory lane quadrant this warp may write
+        const int row = quad * 32 + lane;                        // the four warps of a group cover rows 0..127
         const uint32_t my_bits = bits_ring + (uint32_t)ptid * 16u;
         const bool a16 = (p.cw & 3) == 0;
         const bool plain = (p.kh * p.kw == 1 && p.stride == 1 && p.pad == 0);
@@ -533,12 +569,16 @@ conv_tc_ws_kernel(const ConvProblem p)
             alive = mbar_wait(empty_bar(s), phase, abort_flag, p.err, ERR_PRODUCER_TIMEOUT);
             alive = __all_sync(0xffffffffu, alive);
             if (!alive) break;
-            const uint32_t row_addr = ring + (uint32_t)s * C::A_BYTES + (uint32_t)row * ROWB;
-            expand_store_a(bits.x, row_addr, xr, 0);
-            expand_store_a(bits.y, row_addr, xr, 2);
-            expand_store_a(bits.z, row_addr, xr, 4);
-            expand_store_a(bits.w, row_addr, xr, 6);
-            fence_async_proxy();
+            tc_fence_after();     // the MMAs that read this slot are complete (their commit released it)
+            // expanded row -> 32 columns of this lane: column 8*e + j = word j of K word e (bytes 0 or 2^j)
+            uint32_t v[32];
+            const uint32_t wds[4] = {bits.x, bits.y, bits.z, bits.w};
+#pragma unroll
+            for (int e = 0; e < 4; ++e)
+#pragma unroll
+                for (int j = 0; j < 8; ++j) v[8 * e + j] = wds[e] & (0x01010101u << j);
+            tc_st32(tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(C::A_COL0 + s * 32), v);
+            tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(full_bar(s));
             s += G;
@@ -571,10 +611,9 @@ int launch_ws(const ConvProblem &p0, cudaStream_t stream)
     return cudaGetLastError() == cudaSuccess ? BCNN_OK : BCNN_ERR_CUDA;
 }
 
-// Parity waits are only safe while a waiter is at most one phase behind.  A producer group comes back
-// to the ring every G stages and completion is in order, so the ring must hold at least G stages.
+// The expanded weights, the packed-word staging ring and the tables must fit in shared memory.
 template <int BN, int G>
-bool fits(const ConvProblem &p) { return ws_layout<BN, G>(p.kwords).a_stages >= G; }
+bool fits(const ConvProblem &p) { return ws_layout<BN, G>(p.kwords).smem + 512 <= MAX_SMEM; }
 
 }  // namespace
 
