@@ -71,12 +71,12 @@ int make_conv_problem(ConvProblem &p, const void *x, const void *w, const int32_
 
 // Measured on B200 (bench.py --mode sweep, profiles/engine_bakeoff.md):
 //   * C_out >= 256, or weights too large to keep expanded in shared memory: streaming tcgen05 engine;
-//   * C_out <= 128 with K >= 256 (K >= 128 for C_out > 64): weight-stationary tcgen05 engine;
-//   * shorter K on narrow layers (stem-like 1x1 layers): register-fed warp-level int8 engine;
+//   * C_out <= 128 with K >= 64: weight-stationary tcgen05 engine;
+//   * K = 32 (stem-like 1x1 layer): register-fed warp-level int8 engine;
 //   * the single-bit mma.sync and CUDA-core engines never win and serve as fallbacks.
 int auto_engine(const ConvProblem &p)
 {
-    if (p.C_out <= 128 && p.K >= (p.C_out > 64 ? 128 : 256) && conv_tc_ws_supports(p)) return BCNN_ENGINE_TC_WS;
+    if (p.C_out <= 128 && p.K >= 64 && conv_tc_ws_supports(p)) return BCNN_ENGINE_TC_WS;
     if (p.C_out <= 64 && conv_mma_s8_supports(p)) return BCNN_ENGINE_MMA_S8;
     if (conv_tc_i8_supports(p)) return BCNN_ENGINE_TC_I8;
     if (conv_mma_b1_supports(p)) return BCNN_ENGINE_MMA_B1;

@@ -46,18 +46,22 @@ constexpr int ERR_PRODUCER_TIMEOUT = 111;
 constexpr int ERR_MMA_TIMEOUT = 112;
 constexpr int ERR_EPILOGUE_TIMEOUT = 113;
 
-template <int BN, int G> struct Cfg {
+// DUAL: two CTAs share an SM (two independent MMA issuers), each with half of tensor memory.
+template <int BN, int G, bool DUAL> struct Cfg {
     static constexpr int BNX = BN + 16;                       // + the all-ones row (MMA N is a multiple of 16)
     static constexpr int PROD_THREADS = G * BM;
     static constexpr int CONTROL_WARP = (FIRST_PRODUCER_THREAD + PROD_THREADS) / 32;   // last warp
     static constexpr int THREADS = FIRST_PRODUCER_THREAD + PROD_THREADS + 32;
     // Tensor memory (512 columns): NBUF accumulator buffers of BNX columns, then the activation ring,
     // one stage = 128 rows x 128 expanded bytes = 32 columns.
-    static constexpr int NBUF = BN == 32 ? 4 : (BN == 64 ? 3 : 2);
-    static constexpr int STAGES = BN == 128 ? 7 : 8;
+    static constexpr int TMEM_COLS = DUAL ? 256 : 512;
+    static constexpr int NBUF = DUAL ? 2 : (BN == 32 ? 4 : (BN == 64 ? 3 : 2));
     static constexpr int A_COL0 = NBUF * BNX;
-    static constexpr int TMEM_COLS = 512;
-    static_assert(A_COL0 + STAGES * 32 <= 512, "tensor memory budget");
+    static constexpr int STAGES = (TMEM_COLS - A_COL0) / 32 > 8 ? 8 : (TMEM_COLS - A_COL0) / 32;
+    static constexpr int CTAS_PER_SM = DUAL ? 2 : 1;
+    // registers are granted in blocks of 8 per thread: bound the pair of CTAs to 64 registers per thread
+    static constexpr int BOUND_THREADS = DUAL ? 512 : THREADS;
+    static_assert(A_COL0 + STAGES * 32 <= TMEM_COLS, "tensor memory budget");
     static_assert(STAGES >= G, "a producer group must not lap the ring (parity waits)");
     static constexpr int W_TILE_BYTES = BNX * ROWB;           // one K stage of the expanded weights
     static constexpr int BITS_BYTES = PF * PROD_THREADS * 16;
@@ -244,24 +248,26 @@ struct WsLayout {
     int smem;         // dynamic shared memory in bytes
 };
 
-template <int BN, int G>
+template <int BN, int G, bool DUAL>
 __host__ __device__ inline WsLayout ws_layout(int kwords)
 {
-    using C = Cfg<BN, G>;
+    using C = Cfg<BN, G, DUAL>;
     WsLayout l;
     l.ktiles = (kwords + 3) >> 2;
     l.smem = 1024 + l.ktiles * C::W_TILE_BYTES + C::BITS_BYTES + BN * 4 + l.ktiles * 4 * 4;
-    // each CTA takes all 512 tensor-memory columns: ask for more than half of an SM's shared memory
-    // so that two CTAs of this kernel never share an SM (the second would sit in tcgen05.alloc)
-    if (l.smem < 120 * 1024) l.smem = 120 * 1024;
+    // Tensor memory is shared out by the resident CTAs (all 512 columns, or 256 each for two): ask
+    // for enough shared memory that no further CTA of this kernel fits on the SM (it would sit in
+    // tcgen05.alloc until a neighbour exits).
+    const int floor_bytes = DUAL ? 78 * 1024 : 120 * 1024;
+    if (l.smem < floor_bytes) l.smem = floor_bytes;
     return l;
 }
 
-template <int BN, int G, bool FUSED>
-__global__ void __launch_bounds__(Cfg<BN, G>::THREADS, 1)
+template <int BN, int G, bool DUAL, bool FUSED>
+__global__ void __launch_bounds__(Cfg<BN, G, DUAL>::BOUND_THREADS, Cfg<BN, G, DUAL>::CTAS_PER_SM)
 conv_tc_ws_kernel(const ConvProblem p)
 {
-    using C = Cfg<BN, G>;
+    using C = Cfg<BN, G, DUAL>;
     constexpr int BNX = C::BNX;
     constexpr int NBUF = C::NBUF;
     constexpr int MAX_STAGES = 8;
@@ -273,7 +279,7 @@ conv_tc_ws_kernel(const ConvProblem p)
 
     const int tid = threadIdx.x;
     const int warp = tid >> 5, lane = tid & 31;
-    const WsLayout L = ws_layout<BN, G>(p.kwords);
+    const WsLayout L = ws_layout<BN, G, DUAL>(p.kwords);
     const int ktiles = L.ktiles;
     constexpr int STAGES = C::STAGES;
     const int m_tiles = (p.M + BM - 1) / BM;
@@ -594,7 +600,7 @@ conv_tc_ws_kernel(const ConvProblem p)
     }
 }
 
-template <int BN, int G>
+template <int BN, int G, bool DUAL>
 int launch_ws(const ConvProblem &p0, cudaStream_t stream)
 {
     ConvProblem p = p0;
@@ -602,18 +608,24 @@ int launch_ws(const ConvProblem &p0, cudaStream_t stream)
     int dev = 0, sms = 148;
     cudaGetDevice(&dev);
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    const WsLayout L = ws_layout<BN, G>(p.kwords);
+    using C = Cfg<BN, G, DUAL>;
+    const WsLayout L = ws_layout<BN, G, DUAL>(p.kwords);
     const long m_tiles = ((long)p.M + BM - 1) / BM;
-    const unsigned grid = (unsigned)(m_tiles < sms ? m_tiles : sms);
-    void (*k)(const ConvProblem) = p.thr ? conv_tc_ws_kernel<BN, G, true> : conv_tc_ws_kernel<BN, G, false>;
+    const long slots = (long)sms * C::CTAS_PER_SM;
+    const unsigned grid = (unsigned)(m_tiles < slots ? m_tiles : slots);
+    void (*k)(const ConvProblem) = p.thr ? conv_tc_ws_kernel<BN, G, DUAL, true> : conv_tc_ws_kernel<BN, G, DUAL, false>;
     if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, L.smem) != cudaSuccess) return BCNN_ERR_CUDA;
-    k<<<grid, Cfg<BN, G>::THREADS, L.smem, stream>>>(p);
+    k<<<grid, C::THREADS, L.smem, stream>>>(p);
     return cudaGetLastError() == cudaSuccess ? BCNN_OK : BCNN_ERR_CUDA;
 }
 
-// The expanded weights, the packed-word staging ring and the tables must fit in shared memory.
-template <int BN, int G>
-bool fits(const ConvProblem &p) { return ws_layout<BN, G>(p.kwords).smem + 512 <= MAX_SMEM; }
+// The expanded weights, the packed-word staging ring and the tables must fit in shared memory
+// (in half of it when two CTAs share an SM).
+template <int BN, int G, bool DUAL>
+bool fits(const ConvProblem &p)
+{
+    return ws_layout<BN, G, DUAL>(p.kwords).smem + 512 <= (DUAL ? 113 * 1024 : MAX_SMEM);
+}
 
 }  // namespace
 
@@ -623,18 +635,20 @@ bool conv_tc_ws_supports(const ConvProblem &p)
     if (p.C_out > 128 || p.kh * p.kw > 31 || p.K > (1 << 16)) return false;
     // word offsets of the K-word table are shifted left by 5 bits
     if ((long)(p.kh * (long)p.W + p.kw) * p.cw >= (1L << 26)) return false;
-    if (p.C_out <= 32) return fits<32, 4>(p);
-    if (p.C_out <= 64) return fits<64, 4>(p);
-    return fits<128, 4>(p) || fits<128, 2>(p);
+    if (p.C_out <= 32) return fits<32, 4, false>(p);
+    if (p.C_out <= 64) return fits<64, 4, false>(p);
+    return fits<128, 4, false>(p) || fits<128, 2, false>(p);
 }
 
 int launch_conv_tc_ws(const ConvProblem &p, cudaStream_t stream)
 {
     if (!conv_tc_ws_supports(p)) return BCNN_ERR_UNSUPPORTED;
-    if (p.C_out <= 32) return launch_ws<32, 4>(p, stream);
-    if (p.C_out <= 64) return launch_ws<64, 4>(p, stream);
-    if (fits<128, 4>(p)) return launch_ws<128, 4>(p, stream);
-    return launch_ws<128, 2>(p, stream);     // long K: fewer producer groups leave room for the ring
+    // narrow layers: the per-stage cost of issuing MMAs exceeds their execution time, so two CTAs
+    // per SM (two issuers) when the resident weights leave room for it
+    if (p.C_out <= 32) return fits<32, 2, true>(p) ? launch_ws<32, 2, true>(p, stream) : launch_ws<32, 4, false>(p, stream);
+    if (p.C_out <= 64) return fits<64, 2, true>(p) ? launch_ws<64, 2, true>(p, stream) : launch_ws<64, 4, false>(p, stream);
+    if (fits<128, 4, false>(p)) return launch_ws<128, 4, false>(p, stream);
+    return launch_ws<128, 2, false>(p, stream);     // long K: fewer producer groups, smaller staging ring
 }
 
 }  // namespace bcnn
