@@ -55,7 +55,7 @@ template <int BN, int G, bool DUAL> struct Cfg {
     // Tensor memory (512 columns): NBUF accumulator buffers of BNX columns, then the activation ring,
     // one stage = 128 rows x 128 expanded bytes = 32 columns.
     static constexpr int TMEM_COLS = DUAL ? 256 : 512;
-    static constexpr int NBUF = DUAL ? 2 : (BN == 32 ? 4 : (BN == 64 ? 3 : 2));
+    static constexpr int NBUF = DUAL ? (BN == 128 ? 1 : 2) : (BN == 32 ? 4 : (BN == 64 ? 3 : 2));
     static constexpr int A_COL0 = NBUF * BNX;
     static constexpr int STAGES = (TMEM_COLS - A_COL0) / 32 > 8 ? 8 : (TMEM_COLS - A_COL0) / 32;
     static constexpr int CTAS_PER_SM = DUAL ? 2 : 1;
@@ -647,6 +647,7 @@ int launch_conv_tc_ws(const ConvProblem &p, cudaStream_t stream)
     // per SM (two issuers) when the resident weights leave room for it
     if (p.C_out <= 32) return fits<32, 2, true>(p) ? launch_ws<32, 2, true>(p, stream) : launch_ws<32, 4, false>(p, stream);
     if (p.C_out <= 64) return fits<64, 2, true>(p) ? launch_ws<64, 2, true>(p, stream) : launch_ws<64, 4, false>(p, stream);
+    if (fits<128, 2, true>(p)) return launch_ws<128, 2, true>(p, stream);
     if (fits<128, 4, false>(p)) return launch_ws<128, 4, false>(p, stream);
     return launch_ws<128, 2, false>(p, stream);     // long K: fewer producer groups, smaller staging ring
 }
