@@ -1,213 +1,79 @@
-// Fifth-generation tensor-core engine of the binary implicit GEMM (tcgen05, kind::i8).
+// Streaming tcgen05 engine of the binary implicit GEMM (kind::i8): wide layers (C_out >= 256),
+// long K, and the plain GEMMs.  Arithmetic as in the other tensor-core engines: sign bits are
+// expanded to bytes on chip (activations {0, 2^j}, weights {0, 2^(7-j)}; byte 4j+i of a 32-bit
+// group carries bit j+8i), every product of two set bits is 128, accumulators are int32 in
+// tensor memory and   sum a*g = K - 2*popc(A) - 2*popc(G) + 4*popc(A and G).
 //
-// The tensor cores of sm_100a have no fast single-bit path, so sign bits are expanded
-// to bytes on the fly, in shared memory, and fed to the dense 8-bit integer MMA with
-// int32 accumulators in tensor memory.  Nothing expanded ever touches global memory.
-//
-// Expansion.  Inside every 32-bit group of K the byte at position 4*j + i carries input
-// bit j + 8*i (the sum over K does not care about the order as long as both operands
-// agree).  With that order one 32-bit word of bits w turns into its eight output words
-// with one logic op each:   activations:  w & (0x01010101 << j)         -> byte 0 or 2^j
-//                           weights:      shift(w) & (0x01010101 << 7-j) -> byte 0 or 2^(7-j)
-// so every product of two set bits is exactly 128 and the accumulator holds
-// 128 * popcount(A and G).  With the row / column popcounts,
-//   sum a*g = K - 2*popcount(A) - 2*popcount(G) + 4*popcount(A and G),
-// the popcounts being taken from the words as they are expanded.  Zero words stand for
-// out-of-image taps (value -1), for rows past M, columns past C_out and for the K tail.
-//
-// Persistent, warp-specialised kernel; each CTA walks a static list of 128 x BN tiles.
-//   warp 0        : issues the MMAs (one thread), releases ring slots with tcgen05.commit
-//   warps 1-4     : epilogue - read an accumulator buffer (tcgen05.ld), threshold / pack or
-//                   write int32, hand the buffer back; overlaps the next tile's main loop
-//                   because the accumulators are double-buffered in tensor memory
-//   warps 5...    : producers, one thread per tile row (128 activation rows + BN weight
-//                   rows).  Packed words are staged ahead with cp.async (16 bytes per row
-//                   and stage, zero-filled when out of range), then expanded into a ring of
-//                   128-byte-swizzled K-major tiles, 128 bits of K per stage.
-// Every mbarrier wait is bounded: on expiry the kernel records an error code in the
-// device error word and all roles fall through to the common exit.
-#include "bcnn_common.cuh"
+// Persistent, warp-specialised; each CTA walks a static list of 128 x BN tiles.
+//   warp 0          issuer: tcgen05.mma / commit only, waits on named barriers only (a memory
+//                   instruction after tensor-core instructions would stall it)
+//   warps 1-4       epilogue: tcgen05.ld, threshold + pack (or int32), hand the accumulator back
+//   G = 2 producer groups, each 4 activation warps + BN/32 weight warps, one thread per tile
+//                   row; the groups take the ring's stages alternately so that one group gathers
+//                   while the other expands.  Packed words are staged with cp.async (16 bytes per
+//                   row and stage, zero-fill out of range).
+//                     activation rows -> TENSOR memory (tcgen05.st, 32 columns per stage): the
+//                       MMA takes A from tensor memory, so shared memory carries only weights
+//                     weight rows     -> shared memory, 128-byte-swizzled K-major tiles
+//   last warp       control: does the issuer's mbarrier waits and releases it stage by stage
+// Tensor memory (512 columns): BN = 256: one accumulator + 5 ring stages; BN = 128: two
+// accumulators + 8 ring stages.  Row / column popcounts are taken from the words as they are
+// expanded; each group leaves its partial constants for a tile in shared-memory slots.
+// Every mbarrier wait is bounded and reports through the device error word.
+#include "tc_common.cuh"
 
 namespace bcnn {
 
 namespace {
 
-constexpr int BM = 128;
-constexpr int ROWB = 128;                 // bytes of one expanded tile row per stage (= 128 bits of K)
+using namespace tc;
+
 constexpr int EPI_WARPS = 4;
-constexpr int FIRST_PRODUCER_THREAD = 32 * (1 + EPI_WARPS);
-constexpr uint32_t WAIT_LIMIT = 1u << 17;
-// upper bound (ns) for which one try_wait may suspend the thread: waiting warps then leave
-// the issue slots to the warps that have work; the wake-up on phase completion is immediate
-constexpr uint32_t SUSPEND_HINT_NS = 20000;
+constexpr int G = 2;                      // producer groups
+constexpr int PF = 3;                     // packed-word stages in flight per producer thread
+constexpr int MAX_SMEM = 227 * 1024 - 512; // dynamic shared memory available beside the static part
 
 constexpr int ERR_PRODUCER_TIMEOUT = 101;
 constexpr int ERR_MMA_TIMEOUT = 102;
 constexpr int ERR_EPILOGUE_TIMEOUT = 103;
 
 template <int BN> struct Cfg {
-    static constexpr int PROD_THREADS = BM + BN;
-    static constexpr int THREADS = FIRST_PRODUCER_THREAD + PROD_THREADS;
-    static constexpr int STAGES = BN == 256 ? 4 : (BN == 128 ? 6 : 8);
-    static constexpr int A_BYTES = BM * ROWB;
-    static constexpr int STAGE_BYTES = (BM + BN) * ROWB;
-    static constexpr int SLOTS = STAGES + 3;             // per-tile constant slots: producers run at most STAGES
-                                                         // tiles ahead of the MMAs, the MMAs two tiles ahead of the epilogue
-    static constexpr int PF = BN == 256 ? 3 : 4;         // stages of packed words in flight per producer thread
+    static constexpr int NBUF = BN == 256 ? 1 : 2;                       // accumulator buffers
+    static constexpr int A_COL0 = NBUF * BN;                              // first column of the activation ring
+    static constexpr int STAGES = BN == 256 ? 5 : 8;
+    static constexpr int GROUP_WARPS = 4 + BN / 32;
+    static constexpr int GROUP_THREADS = 32 * GROUP_WARPS;
+    static constexpr int PROD_THREADS = G * GROUP_THREADS;
+    static constexpr int FIRST_PRODUCER_WARP = 1 + EPI_WARPS;
+    static constexpr int CONTROL_WARP = FIRST_PRODUCER_WARP + G * GROUP_WARPS;
+    static constexpr int THREADS = 32 * (CONTROL_WARP + 1);
+    static constexpr int W_BYTES = BN * ROWB;                             // one ring stage of weights
     static constexpr int BITS_BYTES = PF * PROD_THREADS * 16;
-    static constexpr int CONST_BYTES = SLOTS * (BM + BN) * 4;
-    static constexpr int SMEM = 1024 + STAGES * STAGE_BYTES + BITS_BYTES + CONST_BYTES;
-    static constexpr int TMEM_COLS = 2 * BN;             // two accumulator buffers
+    static constexpr int SLOTS = STAGES + NBUF + 2;                       // per-tile constant slots
+    static constexpr int SLOT_INTS = G * (BM + BN);
+    static constexpr int CONST_BYTES = SLOTS * SLOT_INTS * 4;
+    static_assert(A_COL0 + STAGES * 32 <= 512, "tensor memory budget");
+    static_assert(STAGES >= G, "a producer group must not lap the ring (parity waits)");
 };
 
-__device__ __forceinline__ uint32_t smem_u32(const void *p)
-{
-    return static_cast<uint32_t>(__cvta_generic_to_shared(p));
-}
-
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
-{
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
-}
-
-__device__ __forceinline__ void mbar_arrive(uint32_t bar)
-{
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
-{
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok) : "r"(bar), "r"(parity), "r"(SUSPEND_HINT_NS) : "memory");
-    return ok != 0;
-}
-
-// Bounded wait.  Returns false when the limit ran out or another role already gave up.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *err, int code)
-{
-    for (uint32_t it = 0; it < WAIT_LIMIT; ++it) {
-        if (mbar_try_wait(bar, parity)) return true;
-        if ((it & 255u) == 255u && *abort_flag) return false;
-    }
-    *abort_flag = 1;
-    if (err) atomicCAS(err, 0, code);
-    return false;
-}
-
-__device__ __forceinline__ void fence_async_proxy() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-
-__device__ __forceinline__ void tc_commit(uint32_t bar)
-{
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-
-// D[tmem] (+)= A[smem] * B[smem]^T, 8-bit integer operands, int32 accumulators.
-__device__ __forceinline__ void tc_mma_i8(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate)
-{
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, {%5, %6, %7, %8}, p;\n\t}"
-        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(0u), "r"(0u), "r"(0u), "r"(0u)
-        : "memory");
-}
-
-// 32 accumulator columns of this warp's 32 rows.  The load and its completion wait are one asm
-// statement so that no use of the destination registers can be scheduled between them.
-__device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&v)[32])
-{
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-        "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
-        "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];\n\t"
-        "tcgen05.wait::ld.sync.aligned;"
-        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
-          "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
-          "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
-          "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
-        : "r"(taddr) : "memory");
-}
-
-// Shared-memory matrix descriptor of a K-major tile with 128-byte rows and the 128-byte
-// swizzle: 8-row groups are 1024 bytes apart (stride byte offset), descriptor version 1.
-__device__ __forceinline__ uint64_t make_desc(uint32_t saddr)
-{
-    const uint32_t lo = ((saddr & 0x3FFFFu) >> 4) | (1u << 16);
-    const uint32_t hi = (1024u >> 4) | (1u << 14) | (2u << 29);
-    return (static_cast<uint64_t>(hi) << 32) | lo;
-}
-
-// Instruction descriptor: unsigned 8-bit A and B (K-major), int32 accumulate, M = 128, N = BN.
 template <int BN>
-__device__ __forceinline__ constexpr uint32_t make_idesc()
+__host__ __device__ inline int smem_bytes(int ktab_words)
 {
-    return (2u << 4) | (0u << 7) | (0u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
-}
-
-__device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d)
-{
-    asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
-}
-
-__device__ __forceinline__ uint4 ld_shared_v4(uint32_t addr)
-{
-    uint4 v;
-    asm volatile("ld.shared.v4.b32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr) : "memory");
-    return v;
-}
-
-__device__ __forceinline__ void cp_async16(uint32_t dst, const void *src, bool valid)
-{
-    const int n = valid ? 16 : 0;
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(n) : "memory");
-}
-
-__device__ __forceinline__ void cp_async4(uint32_t dst, const void *src, bool valid)
-{
-    const int n = valid ? 4 : 0;
-    asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;" ::"r"(dst), "l"(src), "r"(n) : "memory");
-}
-
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
-template <int N>
-__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
-
-// One word of activation bits -> two 16-byte chunks (bytes 0 or 2^j), stored to chunks c, c+1 of a row.
-__device__ __forceinline__ void expand_store_a(uint32_t w, uint32_t row_addr, int xr, int c)
-{
-    st_shared_v4(row_addr + (uint32_t)(((c) ^ xr) << 4),
-                 w & 0x01010101u, w & 0x02020202u, w & 0x04040404u, w & 0x08080808u);
-    st_shared_v4(row_addr + (uint32_t)(((c + 1) ^ xr) << 4),
-                 w & 0x10101010u, w & 0x20202020u, w & 0x40404040u, w & 0x80808080u);
-}
-
-// One word of weight bits -> two 16-byte chunks (bytes 0 or 2^(7-j)).
-__device__ __forceinline__ void expand_store_w(uint32_t w, uint32_t row_addr, int xr, int c)
-{
-    st_shared_v4(row_addr + (uint32_t)(((c) ^ xr) << 4),
-                 (w << 7) & 0x80808080u, (w << 5) & 0x40404040u, (w << 3) & 0x20202020u, (w << 1) & 0x10101010u);
-    st_shared_v4(row_addr + (uint32_t)(((c + 1) ^ xr) << 4),
-                 (w >> 1) & 0x08080808u, (w >> 3) & 0x04040404u, (w >> 5) & 0x02020202u, (w >> 7) & 0x01010101u);
+    using C = Cfg<BN>;
+    return 1024 + C::STAGES * C::W_BYTES + C::BITS_BYTES + C::CONST_BYTES + ktab_words * 4;
 }
 
 template <int BN, bool FUSED>
 __global__ void __launch_bounds__(Cfg<BN>::THREADS, 1)
-conv_tc_i8_kernel(const ConvProblem p)
+conv_tc_i8_kernel(const ConvProblem p, const int ktab_words)
 {
     using C = Cfg<BN>;
+    constexpr int NBUF = C::NBUF;
     constexpr int STAGES = C::STAGES;
     constexpr int SLOTS = C::SLOTS;
-    constexpr int PT = C::PROD_THREADS;
-    constexpr int PF = C::PF;
 
     extern __shared__ unsigned char smem_raw[];
-    __shared__ __align__(8) unsigned long long bars[2 * STAGES + 4];
+    __shared__ __align__(8) unsigned long long bars[2 * 8 + 2 * 2];
     __shared__ uint32_t tmem_base_smem;
     __shared__ int abort_flag_smem;
 
@@ -218,20 +84,22 @@ conv_tc_i8_kernel(const ConvProblem p)
     const int n_tiles = (p.C_out + BN - 1) / BN;
     const int total_tiles = m_tiles * n_tiles;
     const int my_tiles = ((int)blockIdx.x < total_tiles) ? (total_tiles - 1 - (int)blockIdx.x) / (int)gridDim.x + 1 : 0;
+    const int total_items = my_tiles * ktiles;
 
-    const uint32_t ring = (smem_u32(smem_raw) + 1023u) & ~1023u;
-    const uint32_t bits_ring = ring + STAGES * C::STAGE_BYTES;
-    const uint32_t consts = bits_ring + C::BITS_BYTES;        // [SLOTS][BM + BN] int32
+    const uint32_t wring = (smem_u32(smem_raw) + 1023u) & ~1023u;         // [STAGES][BN rows][128 B]
+    const uint32_t bits_ring = wring + STAGES * C::W_BYTES;               // [PF][PROD_THREADS][16 B]
+    const uint32_t consts = bits_ring + C::BITS_BYTES;                    // [SLOTS][G][BM + BN] int32
+    const uint32_t ktab_addr = consts + C::CONST_BYTES;                   // [ktab_words] (word offset << 5) | tap
     const uint32_t bar0 = smem_u32(bars);
     auto full_bar = [&](int s) { return bar0 + 8u * s; };
-    auto empty_bar = [&](int s) { return bar0 + 8u * (STAGES + s); };
-    auto tfull_bar = [&](int b) { return bar0 + 8u * (2 * STAGES + b); };
-    auto tempty_bar = [&](int b) { return bar0 + 8u * (2 * STAGES + 2 + b); };
+    auto empty_bar = [&](int s) { return bar0 + 8u * (8 + s); };
+    auto tfull_bar = [&](int b) { return bar0 + 8u * (16 + b); };
+    auto tempty_bar = [&](int b) { return bar0 + 8u * (18 + b); };
     volatile int *abort_flag = &abort_flag_smem;
 
     if (tid == 0) {
-        for (int s = 0; s < STAGES; ++s) {
-            mbar_init(full_bar(s), PT / 32);      // one arrival per producer warp
+        for (int s = 0; s < 8; ++s) {
+            mbar_init(full_bar(s), C::GROUP_WARPS);      // every warp of the group that owns the stage
             mbar_init(empty_bar(s), 1);
         }
         for (int b = 0; b < 2; ++b) {
@@ -242,8 +110,17 @@ conv_tc_i8_kernel(const ConvProblem p)
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 0) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_smem)), "r"((uint32_t)C::TMEM_COLS) : "memory");
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_smem)), "r"(512u) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    for (int kword = tid; kword < ktab_words; kword += C::THREADS) {
+        int entry = 31;                          // tap 31 is never valid (at most 31 taps)
+        if (kword < p.kwords) {
+            const int tap = kword / p.cw, cj = kword - tap * p.cw;
+            const int r = tap / p.kw, t = tap - r * p.kw;
+            entry = (((r * p.W + t) * p.cw + cj) << 5) | tap;
+        }
+        asm volatile("st.shared.b32 [%0], %1;" ::"r"(ktab_addr + 4u * kword), "r"(entry) : "memory");
     }
     tc_fence_before();
     __syncthreads();
@@ -251,54 +128,84 @@ conv_tc_i8_kernel(const ConvProblem p)
     const uint32_t tmem_base = tmem_base_smem;
 
     if (warp == 0) {
-        // ------------------------------------------------------------------ MMA issuer
-        if (lane == 0) {
-            constexpr uint32_t idesc = make_idesc<BN>();
-            int s = 0;
-            uint32_t ring_phase = 0;
-            bool alive = true;
-            for (int ti = 0; ti < my_tiles && alive; ++ti) {
-                const int buf = ti & 1;
-                alive = mbar_wait(tempty_bar(buf), ((ti >> 1) & 1) ^ 1, abort_flag, p.err, ERR_MMA_TIMEOUT);
-                if (!alive) break;
+        // ------------------------------------------------------------------ issuer (no memory instructions)
+        constexpr uint32_t idesc = make_idesc(BN);
+        const uint64_t desc0 = make_desc(0);
+        const uint32_t desc_hi = (uint32_t)(desc0 >> 32);
+        const uint32_t b_lo0 = (uint32_t)desc0 | ((wring & 0x3FFFFu) >> 4);      // + slot * (W_BYTES / 16)
+        const uint32_t a_tmem0 = tmem_base + (uint32_t)C::A_COL0;                // + slot * 32 columns
+        const uint32_t elected = lane == 0 ? 1u : 0u;
+        int s = 0, buf = 0;
+        for (int ti = 0; ti < my_tiles; ++ti) {
+            const uint32_t d_tmem = tmem_base + (uint32_t)(buf * BN);
+            const uint32_t tfull = tfull_bar(buf);
+            for (int kt = 0; kt < ktiles; ++kt) {
+                const uint32_t a_t = a_tmem0 + (uint32_t)s * 32u;
+                const uint32_t b_lo = b_lo0 + (uint32_t)s * (C::W_BYTES >> 4);
+                const int nk = p.kwords - 4 * kt;                 // 32 bits of K per instruction; skip the zero tail
+                const uint32_t e1 = nk > 1 ? elected : 0u, e2 = nk > 2 ? elected : 0u, e3 = nk > 3 ? elected : 0u;
+                const uint32_t last = (kt == ktiles - 1) ? elected : 0u;
+                const uint32_t ebar = empty_bar(s);
+                asm volatile("bar.sync %0, 64;" ::"r"(1 + s) : "memory");
                 tc_fence_after();
-                const uint32_t d_tmem = tmem_base + (uint32_t)(buf * BN);
-                for (int kt = 0; kt < ktiles; ++kt) {
-                    alive = mbar_wait(full_bar(s), ring_phase, abort_flag, p.err, ERR_MMA_TIMEOUT);
-                    if (!alive) break;
-                    tc_fence_after();
-                    const uint32_t a_tile = ring + (uint32_t)s * C::STAGE_BYTES;
-                    const uint64_t a_desc = make_desc(a_tile);
-                    const uint64_t b_desc = make_desc(a_tile + C::A_BYTES);
-#pragma unroll
-                    for (int k = 0; k < 4; ++k)   // 32 bytes of K per instruction: +2 in 16-byte address units
-                        tc_mma_i8(d_tmem, a_desc + 2u * k, b_desc + 2u * k, idesc, (kt > 0 || k > 0) ? 1u : 0u);
-                    tc_commit(empty_bar(s));
-                    if (++s == STAGES) { s = 0; ring_phase ^= 1u; }
-                }
-                if (alive) tc_commit(tfull_bar(buf));
+                // per 32 bytes of K: 8 tensor-memory columns of A, +2 (16-byte units) in the B descriptor
+                tc_mma_i8_ts_pred(d_tmem, a_t, b_lo, desc_hi, idesc, kt > 0 ? 1u : 0u, elected);
+                tc_mma_i8_ts_pred(d_tmem, a_t + 8u, b_lo + 2u, desc_hi, idesc, 1u, e1);
+                tc_mma_i8_ts_pred(d_tmem, a_t + 16u, b_lo + 4u, desc_hi, idesc, 1u, e2);
+                tc_mma_i8_ts_pred(d_tmem, a_t + 24u, b_lo + 6u, desc_hi, idesc, 1u, e3);
+                tc_commit_pred(ebar, elected);
+                tc_commit_pred(tfull, last);
+                if (++s == STAGES) s = 0;
             }
+            if (++buf == NBUF) buf = 0;
         }
-        __syncwarp();
+    } else if (warp == C::CONTROL_WARP) {
+        // ------------------------------------------------------------------ control: waits for the issuer
+        // A stage is released (bar.arrive on 1 + slot) once its ring slot is full and, for a tile's
+        // first stage, once the accumulator buffer is free.  The slot being full implies that the
+        // issuer is past the previous use of the same named barrier.  After a time-out the remaining
+        // stages are released without waiting so that the issuer always terminates.
+        int s = 0, buf = 0;
+        uint32_t ring_phase = 0, buf_phase = 1;      // first use of every accumulator buffer: free
+        bool alive = true;
+        for (int ti = 0; ti < my_tiles; ++ti) {
+            if (lane == 0 && alive) alive = mbar_wait(tempty_bar(buf), buf_phase, abort_flag, p.err, ERR_MMA_TIMEOUT);
+            for (int kt = 0; kt < ktiles; ++kt) {
+                if (lane == 0 && alive) alive = mbar_wait(full_bar(s), ring_phase, abort_flag, p.err, ERR_MMA_TIMEOUT);
+                __syncwarp();
+                asm volatile("bar.arrive %0, 64;" ::"r"(1 + s) : "memory");
+                if (++s == STAGES) { s = 0; ring_phase ^= 1u; }
+            }
+            if (++buf == NBUF) { buf = 0; buf_phase ^= 1u; }
+        }
     } else if (warp <= EPI_WARPS) {
         // ------------------------------------------------------------------ epilogue
         const int quad = warp & 3;                 // tensor-memory lane quadrant this warp may read
         const int erow = quad * 32 + lane;
         bool alive = true;
+        int buf = 0;
+        uint32_t buf_phase = 0;
         for (int ti = 0; ti < my_tiles; ++ti) {
             const int tile = (int)blockIdx.x + ti * (int)gridDim.x;
             const int n_tile = tile / m_tiles, m_tile = tile - n_tile * m_tiles;
             const int m0 = m_tile * BM, n0 = n_tile * BN;
-            const int buf = ti & 1;
-            const uint32_t slot = consts + (uint32_t)((ti % SLOTS) * (BM + BN) * 4);
-            if (alive) alive = mbar_wait(tfull_bar(buf), (ti >> 1) & 1, abort_flag, p.err, ERR_EPILOGUE_TIMEOUT);
+            const int em = m0 + erow;
+            // which producer groups took part in this tile (each leaves partial constants): both,
+            // unless the tile is a single stage
+            const int first_group = (ti * ktiles) & 1;
+            const bool two = ktiles >= 2;
+            const uint32_t slot = consts + (uint32_t)((ti % SLOTS) * C::SLOT_INTS * 4);
+            const uint32_t part0 = slot + (uint32_t)(first_group * (BM + BN) * 4);
+            const uint32_t part1 = slot + (uint32_t)((first_group ^ 1) * (BM + BN) * 4);
+            if (alive) alive = mbar_wait(tfull_bar(buf), buf_phase, abort_flag, p.err, ERR_EPILOGUE_TIMEOUT);
             alive = __all_sync(0xffffffffu, alive && !*abort_flag);
             if (!alive) break;
             tc_fence_after();
-            const int em = m0 + erow;
-            int rowc;
-            asm volatile("ld.shared.b32 %0, [%1];" : "=r"(rowc) : "r"(slot + 4u * erow) : "memory");
-            const uint32_t colc_addr = slot + 4u * BM;
+            int rowc, rowc1 = 0;
+            asm volatile("ld.shared.b32 %0, [%1];" : "=r"(rowc) : "r"(part0 + 4u * erow) : "memory");
+            if (two) asm volatile("ld.shared.b32 %0, [%1];" : "=r"(rowc1) : "r"(part1 + 4u * erow) : "memory");
+            rowc += rowc1;
+            const uint32_t c0_addr = part0 + 4u * BM, c1_addr = part1 + 4u * BM;
             const uint32_t t_addr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(buf * BN);
             uint32_t words[BN / 32];
 #pragma unroll
@@ -309,11 +216,15 @@ conv_tc_i8_kernel(const ConvProblem p)
                     uint32_t v[32];
                     tc_ld32(t_addr + (uint32_t)col0, v);
                     if (FUSED) {
-                        // bit = (v + rowc + colc >= 0); sign bits are shifted in last column first
+                        // bit = (v + rowc + colc >= 0); sign bits are shifted in, last column first
                         uint32_t acc = 0;
 #pragma unroll
                         for (int i4 = 7; i4 >= 0; --i4) {
-                            const uint4 cc = ld_shared_v4(colc_addr + 4u * (col0 + 4 * i4));
+                            uint4 cc = ld_shared_v4(c0_addr + 4u * (col0 + 4 * i4));
+                            if (two) {
+                                const uint4 c2 = ld_shared_v4(c1_addr + 4u * (col0 + 4 * i4));
+                                cc.x += c2.x; cc.y += c2.y; cc.z += c2.z; cc.w += c2.w;
+                            }
                             acc = __funnelshift_l((uint32_t)((int)v[4 * i4 + 3] + rowc + (int)cc.w), acc, 1);
                             acc = __funnelshift_l((uint32_t)((int)v[4 * i4 + 2] + rowc + (int)cc.z), acc, 1);
                             acc = __funnelshift_l((uint32_t)((int)v[4 * i4 + 1] + rowc + (int)cc.y), acc, 1);
@@ -325,7 +236,11 @@ conv_tc_i8_kernel(const ConvProblem p)
                         const bool vec = (p.C_out & 3) == 0 && (n0 + col0 + 32 <= p.C_out);
 #pragma unroll
                         for (int i4 = 0; i4 < 8; ++i4) {
-                            const uint4 cc = ld_shared_v4(colc_addr + 4u * (col0 + 4 * i4));
+                            uint4 cc = ld_shared_v4(c0_addr + 4u * (col0 + 4 * i4));
+                            if (two) {
+                                const uint4 c2 = ld_shared_v4(c1_addr + 4u * (col0 + 4 * i4));
+                                cc.x += c2.x; cc.y += c2.y; cc.z += c2.z; cc.w += c2.w;
+                            }
                             int4 o;
                             o.x = (int)(v[4 * i4 + 0] >> 5) + rowc + (int)cc.x;
                             o.y = (int)(v[4 * i4 + 1] >> 5) + rowc + (int)cc.y;
@@ -344,14 +259,15 @@ conv_tc_i8_kernel(const ConvProblem p)
                     }
                 }
             }
-            // all reads of this accumulator buffer are complete: hand it back to the MMA warp
+            // all reads of this accumulator buffer are complete: hand it back
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(tempty_bar(buf));
+            if (++buf == NBUF) { buf = 0; buf_phase ^= 1u; }
             if (FUSED && em < p.M) {
                 const int owords = p.C_out >> 5;
                 uint32_t *dst = static_cast<uint32_t *>(p.out) + (long)em * owords + (n0 >> 5);
-                if (BN >= 128 && (owords & 3) == 0 && n0 + BN <= p.C_out) {
+                if ((owords & 3) == 0 && n0 + BN <= p.C_out) {
 #pragma unroll
                     for (int c4 = 0; c4 < BN / 128; ++c4)
                         *reinterpret_cast<uint4 *>(dst + 4 * c4) =
@@ -365,149 +281,155 @@ conv_tc_i8_kernel(const ConvProblem p)
         }
     } else {
         // ------------------------------------------------------------------ producers
-        const int ptid = tid - FIRST_PRODUCER_THREAD;
-        const bool is_a = ptid < BM;
-        const int row = is_a ? ptid : ptid - BM;                 // row inside the A or the W tile
-        const int xr = row & 7;                                  // swizzle term of this row
-        const uint32_t row_off = (is_a ? 0u : (uint32_t)C::A_BYTES) + (uint32_t)row * ROWB;
+        const int pw = warp - C::FIRST_PRODUCER_WARP;            // producer warp index
+        const int grp = pw / C::GROUP_WARPS, gw = pw - grp * C::GROUP_WARPS;
+        const bool is_a = gw < 4;
+        // activation warps are matched to tensor-memory lane quadrants (a warp may only touch
+        // lanes 32 * (warp % 4) ...): the first four warps of a group have four distinct residues
+        const int quad = warp & 3;
+        const int row = is_a ? quad * 32 + lane : (gw - 4) * 32 + lane;   // row of the A or of the W tile
+        const int ptid = tid - 32 * C::FIRST_PRODUCER_WARP;
+        const int crow = is_a ? row : BM + row;                  // index into a constants part
         const uint32_t my_bits = bits_ring + (uint32_t)ptid * 16u;
-        const bool a16 = (p.cw & 3) == 0;                        // a stage never straddles two taps
+        const bool a16 = (p.cw & 3) == 0;
         const bool w16 = (p.kwords & 3) == 0;
-        const int total_items = my_tiles * ktiles;
+        const bool plain = (p.kh * p.kw == 1 && p.stride == 1 && p.pad == 0);
 
-        // ---- load cursor (runs PF - 1 items ahead of the expand cursor)
-        int l_ti = 0, l_kt = 0, l_r = 0, l_t = 0, l_cj = 0, l_slot = 0;
-        bool l_ok = false;
+        // this thread's items: grp, grp + G, ... of the CTA's flattened (tile, stage) list
+        // ---- load cursor
+        int l_it = grp, l_ti = 0, l_kt = grp, l_slot = 0;
+        bool l_fresh = true;
         const uint32_t *l_base = p.x;
-        int l_ih0 = 0, l_iw0 = 0;
-        auto l_new_tile = [&]() {
-            const int tile = (int)blockIdx.x + l_ti * (int)gridDim.x;
-            const int n_tile = tile / m_tiles, m_tile = tile - n_tile * m_tiles;
-            if (is_a) {
-                const int m = m_tile * BM + row;
-                l_ok = m < p.M;
-                const RowCoord rc = row_coord(p, l_ok ? m : 0);
-                l_base = p.x + (long)rc.b * p.H * p.W * p.cw;
-                l_ih0 = rc.ih0;
-                l_iw0 = rc.iw0;
-            } else {
-                const int n = n_tile * BN + row;
-                l_ok = n < p.C_out;
-                l_base = p.w + (long)(l_ok ? n : 0) * p.kwords;
+        uint32_t l_mask = 0;
+        auto l_locate = [&]() {
+            while (l_kt >= ktiles) { l_kt -= ktiles; ++l_ti; l_fresh = true; }
+            if (l_fresh) {
+                l_fresh = false;
+                const int tile = (int)blockIdx.x + l_ti * (int)gridDim.x;
+                const int n_tile = tile / m_tiles, m_tile = tile - n_tile * m_tiles;
+                if (is_a) {
+                    const int m = m_tile * BM + row;
+                    const bool ok = m < p.M;
+                    if (plain) {
+                        l_base = p.x + (long)(ok ? m : 0) * p.cw;
+                        l_mask = ok ? 1u : 0u;
+                    } else {
+                        const RowCoord rc = row_coord(p, ok ? m : 0);
+                        l_base = p.x + (((long)rc.b * p.H + rc.ih0) * p.W + rc.iw0) * p.cw;
+                        uint32_t colbits = 0, mask = 0;
+                        for (int t = 0; t < p.kw; ++t)
+                            if (rc.iw0 + t >= 0 && rc.iw0 + t < p.W) colbits |= 1u << t;
+                        for (int r = 0; r < p.kh; ++r)
+                            if (rc.ih0 + r >= 0 && rc.ih0 + r < p.H) mask |= colbits << (r * p.kw);
+                        l_mask = ok ? mask : 0u;
+                    }
+                } else {
+                    const int n = n_tile * BN + row;
+                    const bool ok = n < p.C_out;
+                    l_base = p.w + (long)(ok ? n : 0) * p.kwords;
+                    l_mask = ok ? 1u : 0u;
+                }
             }
-            l_kt = 0; l_r = 0; l_t = 0; l_cj = 0;
         };
         auto issue_load = [&]() {
-            const uint32_t dst = my_bits + (uint32_t)l_slot * (PT * 16u);
-            if (is_a) {
-                if (a16) {
-                    const int ih = l_ih0 + l_r, iw = l_iw0 + l_t;
-                    const bool ok = l_ok && ih >= 0 && ih < p.H && iw >= 0 && iw < p.W;
-                    cp_async16(dst, ok ? l_base + ((long)ih * p.W + iw) * p.cw + l_cj : p.x, ok);
-                    l_cj += 4;
-                    if (l_cj == p.cw) {
-                        l_cj = 0;
-                        if (++l_t == p.kw) { l_t = 0; ++l_r; }
-                    }
+            l_locate();
+            const uint32_t dst = my_bits + (uint32_t)l_slot * (C::PROD_THREADS * 16u);
+            if (!is_a || plain) {
+                // contiguous K: word kt*4 + e of the row
+                const bool rok = l_mask != 0;
+                if (is_a ? a16 : w16) {
+                    cp_async16(dst, rok ? l_base + l_kt * 4 : p.x, rok);
                 } else {
 #pragma unroll
                     for (int e = 0; e < 4; ++e) {
                         const int kword = l_kt * 4 + e;
-                        bool ok = l_ok && kword < p.kwords;
-                        const uint32_t *src = p.x;
-                        if (ok) {
-                            const int tap = fast_div(kword, p.cw_magic);
-                            const int cj = kword - tap * p.cw;
-                            const int r = fast_div(tap, p.kw_magic);
-                            const int t = tap - r * p.kw;
-                            const int ih = l_ih0 + r, iw = l_iw0 + t;
-                            ok = ih >= 0 && ih < p.H && iw >= 0 && iw < p.W;
-                            if (ok) src = l_base + ((long)ih * p.W + iw) * p.cw + cj;
-                        }
-                        cp_async4(dst + 4u * e, src, ok);
+                        const bool ok = rok && kword < p.kwords;
+                        cp_async4(dst + 4u * e, ok ? l_base + kword : p.x, ok);
                     }
                 }
+            } else if (a16) {
+                int entry;
+                asm volatile("ld.shared.b32 %0, [%1];" : "=r"(entry) : "r"(ktab_addr + 16u * l_kt));
+                const bool ok = (l_mask >> (entry & 31)) & 1u;
+                cp_async16(dst, ok ? l_base + (entry >> 5) : p.x, ok);
             } else {
-                if (w16) {
-                    cp_async16(dst, l_ok ? l_base + l_kt * 4 : p.w, l_ok);
-                } else {
+                const uint4 e4 = ld_shared_v4(ktab_addr + 16u * l_kt);
+                const int ent[4] = {(int)e4.x, (int)e4.y, (int)e4.z, (int)e4.w};
 #pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        const int kword = l_kt * 4 + e;
-                        const bool ok = l_ok && kword < p.kwords;
-                        cp_async4(dst + 4u * e, ok ? l_base + kword : p.w, ok);
-                    }
+                for (int e = 0; e < 4; ++e) {
+                    const bool ok = (l_mask >> (ent[e] & 31)) & 1u;
+                    cp_async4(dst + 4u * e, ok ? l_base + (ent[e] >> 5) : p.x, ok);
                 }
             }
-            if (++l_kt == ktiles) {
-                ++l_ti;
-                if (l_ti < my_tiles) l_new_tile();
-            }
+            l_it += G;
+            l_kt += G;
             if (++l_slot == PF) l_slot = 0;
         };
 
-        if (my_tiles > 0) l_new_tile();
-        int issued = 0;
 #pragma unroll 1
-        for (; issued < PF - 1; ++issued) {
-            if (issued < total_items) issue_load();
+        for (int i = 0; i < PF - 1; ++i) {
+            if (l_it < total_items) issue_load();
             cp_async_commit();
         }
 
         // ---- expand cursor
-        int s = 0, c_slot = 0, c_kt = 0, c_ti = 0, pop = 0;
-        uint32_t ring_phase = 1;             // first pass through the ring: slots are free
-        int thr_n = 0;
-        bool n_ok = false;
-        auto c_new_tile = [&]() {
-            if (!is_a) {
-                const int tile = (int)blockIdx.x + c_ti * (int)gridDim.x;
-                const int n = (tile / m_tiles) * BN + row;
-                n_ok = n < p.C_out;
-                thr_n = (FUSED && n_ok) ? __ldg(p.thr + n) : 0;
-            }
-        };
-        if (my_tiles > 0) c_new_tile();
+        int c_slot = 0, c_ti = 0, c_kt = grp, pop = 0;
+        int s = grp;
+        uint32_t phase = 1;                   // first pass through the ring: slots are free
+        while (s >= STAGES) { s -= STAGES; phase ^= 1u; }
         bool alive = true;
-        for (int it = 0; it < total_items; ++it) {
-            if (issued < total_items) issue_load();
-            ++issued;
+        for (int it = grp; it < total_items; it += G) {
+            if (l_it < total_items) issue_load();
             cp_async_commit();
             cp_async_wait<PF - 1>();
-            const uint4 bits = ld_shared_v4(my_bits + (uint32_t)c_slot * (PT * 16u));
+            const uint4 bits = ld_shared_v4(my_bits + (uint32_t)c_slot * (C::PROD_THREADS * 16u));
             if (++c_slot == PF) c_slot = 0;
-            alive = mbar_wait(empty_bar(s), ring_phase, abort_flag, p.err, ERR_PRODUCER_TIMEOUT);
+            while (c_kt >= ktiles) { c_kt -= ktiles; ++c_ti; }
+            alive = mbar_wait(empty_bar(s), phase, abort_flag, p.err, ERR_PRODUCER_TIMEOUT);
             alive = __all_sync(0xffffffffu, alive);
             if (!alive) break;
-            const uint32_t row_addr = ring + (uint32_t)s * C::STAGE_BYTES + row_off;
+            pop += __popc(bits.x) + __popc(bits.y) + __popc(bits.z) + __popc(bits.w);
+            if (c_kt + G >= ktiles) {
+                // this group's last stage of the tile: leave its partial constants for the epilogue.
+                //   fused: bit = acc - 64*pa - 32*(thr - K + 2*pg) >= 0      int32: (acc >> 5) - 2*pa + K - 2*pg
+                // the term that does not depend on the popcounts goes with the group of the tile's first stage
+                const bool first_group = ((c_ti * ktiles) & 1) == grp;
+                int cst = FUSED ? -64 * pop : -2 * pop;
+                if (!is_a && first_group) {
+                    const int tile = (int)blockIdx.x + c_ti * (int)gridDim.x;
+                    const int n = (tile / m_tiles) * BN + row;
+                    const int thr_n = (FUSED && n < p.C_out) ? __ldg(p.thr + n) : 0;
+                    cst += FUSED ? -32 * (thr_n - p.K) : p.K;
+                }
+                const uint32_t part = consts + (uint32_t)(((c_ti % SLOTS) * C::SLOT_INTS + grp * (BM + BN) + crow) * 4);
+                asm volatile("st.shared.b32 [%0], %1;" ::"r"(part), "r"(cst) : "memory");
+                pop = 0;
+            }
             if (is_a) {
-                expand_store_a(bits.x, row_addr, xr, 0);
-                expand_store_a(bits.y, row_addr, xr, 2);
-                expand_store_a(bits.z, row_addr, xr, 4);
-                expand_store_a(bits.w, row_addr, xr, 6);
+                tc_fence_after();     // the MMAs that read this slot are complete (their commit released it)
+                // expanded row -> 32 columns of this lane: column 8*e + j = word j of K word e (bytes 0 or 2^j)
+                uint32_t v[32];
+                const uint32_t wds[4] = {bits.x, bits.y, bits.z, bits.w};
+#pragma unroll
+                for (int e = 0; e < 4; ++e)
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) v[8 * e + j] = wds[e] & (0x01010101u << j);
+                tc_st32(tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(C::A_COL0 + s * 32), v);
+                tc_fence_before();
             } else {
+                const uint32_t row_addr = wring + (uint32_t)s * C::W_BYTES + (uint32_t)row * ROWB;
+                const int xr = row & 7;
                 expand_store_w(bits.x, row_addr, xr, 0);
                 expand_store_w(bits.y, row_addr, xr, 2);
                 expand_store_w(bits.z, row_addr, xr, 4);
                 expand_store_w(bits.w, row_addr, xr, 6);
+                fence_async_proxy();  // generic-proxy stores -> visible to the MMA (async proxy)
             }
-            pop += __popc(bits.x) + __popc(bits.y) + __popc(bits.z) + __popc(bits.w);
-            if (++c_kt == ktiles) {
-                // per-tile constants of this row / column, read by the epilogue of this tile
-                int cst;
-                if (is_a) cst = FUSED ? -64 * pop : -2 * pop;
-                else      cst = FUSED ? -32 * (thr_n - p.K + 2 * pop) : p.K - 2 * pop;
-                const uint32_t slot = consts + (uint32_t)((c_ti % SLOTS) * (BM + BN) * 4);
-                asm volatile("st.shared.b32 [%0], %1;" ::"r"(slot + 4u * ptid), "r"(cst) : "memory");
-                pop = 0;
-                c_kt = 0;
-                ++c_ti;
-                if (c_ti < my_tiles) c_new_tile();
-            }
-            fence_async_proxy();          // make this thread's generic-proxy stores visible to the MMA (async proxy)
             __syncwarp();
             if (lane == 0) mbar_arrive(full_bar(s));
-            if (++s == STAGES) { s = 0; ring_phase ^= 1u; }
+            s += G;
+            while (s >= STAGES) { s -= STAGES; phase ^= 1u; }
+            c_kt += G;
         }
         cp_async_wait<0>();
     }
@@ -515,8 +437,14 @@ conv_tc_i8_kernel(const ConvProblem p)
     tc_fence_before();
     __syncthreads();
     if (warp == 0) {
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"((uint32_t)C::TMEM_COLS) : "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512u) : "memory");
     }
+}
+
+int ktab_words_for(const ConvProblem &p)
+{
+    const bool plain = (p.kh * p.kw == 1 && p.stride == 1 && p.pad == 0);
+    return plain ? 0 : ((p.kwords + 3) & ~3);
 }
 
 template <int BN>
@@ -532,19 +460,11 @@ int launch_bn(const ConvProblem &p0, cudaStream_t stream)
     const long total = m_tiles * n_tiles;
     if (total >= (1L << 31)) return BCNN_ERR_UNSUPPORTED;
     const unsigned grid = (unsigned)(total < sms ? total : sms);
-    const int smem = Cfg<BN>::SMEM;
-    cudaError_t e;
-    if (p.thr) {
-        auto k = conv_tc_i8_kernel<BN, true>;
-        e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-        if (e != cudaSuccess) return BCNN_ERR_CUDA;
-        k<<<grid, Cfg<BN>::THREADS, smem, stream>>>(p);
-    } else {
-        auto k = conv_tc_i8_kernel<BN, false>;
-        e = cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
-        if (e != cudaSuccess) return BCNN_ERR_CUDA;
-        k<<<grid, Cfg<BN>::THREADS, smem, stream>>>(p);
-    }
+    const int ktw = ktab_words_for(p);
+    const int smem = smem_bytes<BN>(ktw);
+    void (*k)(const ConvProblem, const int) = p.thr ? conv_tc_i8_kernel<BN, true> : conv_tc_i8_kernel<BN, false>;
+    if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return BCNN_ERR_CUDA;
+    k<<<grid, Cfg<BN>::THREADS, smem, stream>>>(p, ktw);
     return cudaGetLastError() == cudaSuccess ? BCNN_OK : BCNN_ERR_CUDA;
 }
 
@@ -553,16 +473,20 @@ int launch_bn(const ConvProblem &p0, cudaStream_t stream)
 bool conv_tc_i8_supports(const ConvProblem &p)
 {
     if (p.thr != nullptr && (p.C_out % 32 != 0)) return false;
-    // the multiplier-based divisions need kword * cw < 2^32 and the epilogue constants (3K << 5) < 2^31
+    if (p.kh * p.kw > 31) return false;                       // one validity bit per tap
+    if ((long)(p.kh * (long)p.W + p.kw) * p.cw >= (1L << 26)) return false;   // table offsets are shifted by 5 bits
+    if (smem_bytes<256>(ktab_words_for(p)) > MAX_SMEM) return false;   // the K-word table of the gather must fit
+    // the epilogue constants (about 3K << 5) must stay below 2^31
     return p.K <= (1 << 20);
 }
 
 int launch_conv_tc_i8(const ConvProblem &p, cudaStream_t stream)
 {
     if (!conv_tc_i8_supports(p)) return BCNN_ERR_UNSUPPORTED;
-    if (p.C_out > 128) return launch_bn<256>(p, stream);
-    if (p.C_out > 64) return launch_bn<128>(p, stream);
-    return launch_bn<64>(p, stream);
+    // 256-wide tiles have a single accumulator buffer (tensor memory also holds the activation
+    // ring), so their epilogue is not overlapped: worth it only when the K loop is long
+    if (p.C_out > 128 && p.kwords >= 24) return launch_bn<256>(p, stream);
+    return launch_bn<128>(p, stream);
 }
 
 }  // namespace bcnn
