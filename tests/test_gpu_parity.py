@@ -176,6 +176,31 @@ def test_pack(bk, oracle, shape):
     assert np.array_equal(synth.unpack_bits(out.cpu().numpy().reshape(B, H, W, C // 8)), want)
 
 
+def test_pack_stem_nonfinite_and_tied_biases(bk, oracle):
+    # stem shape (4 real channels x 8): infinite / NaN biases take the per-channel path
+    # (inf + -inf = NaN -> -1), equal biases exercise ties in the sorted-threshold path
+    rng = np.random.default_rng(4242)
+    B, H, W = 2, 9, 11
+    x = synth.real_input(rng, (B, H, W, 4))
+    x.reshape(-1)[:12] = [0.0, -0.0, np.inf, -np.inf, np.nan, 1e-45, -1e-45, 0.5, -0.5, 1.0, -1.0, 2.0]
+    for kind in ("inf", "nan", "ties", "zeros"):
+        bias = synth.real_input(rng, (32,))
+        if kind == "inf":
+            bias[3], bias[10] = np.inf, -np.inf
+        elif kind == "nan":
+            bias[7] = np.nan
+        elif kind == "ties":
+            bias[:] = np.repeat(np.array([0.5, -0.5, 0.0, -0.0], np.float32), 8)
+            bias[5] = -x.reshape(-1)[21]           # exact tie x + b == 0 on one channel
+        else:
+            bias[:] = 0.0
+        want = oracle.binarize(x, bias, 8)
+        out = torch.empty(B * H * W * 4, dtype=torch.uint8, device="cuda")
+        bk.bcnn_pack(dev(x), dev(bias), out, B, H, W, 4, 8)
+        torch.cuda.synchronize()
+        assert np.array_equal(synth.unpack_bits(out.cpu().numpy().reshape(B, H, W, 4)), want), kind
+
+
 def test_pack_weights_layout(bk, oracle):
     # packing real weights [C_out][kh][kw][C_in] with the same call gives the conv weight layout
     rng = np.random.default_rng(77)
