@@ -71,11 +71,13 @@ int make_conv_problem(ConvProblem &p, const void *x, const void *w, const int32_
 
 // Measured on B200 (bench.py --mode sweep, profiles/engine_bakeoff.md):
 //   * C_out >= 256, or weights too large to keep expanded in shared memory: streaming tcgen05 engine;
+//   * 1x1 layer with C_in = 32 and C_out <= 32 (one XOR + popcount per output): CUDA-core pointwise kernel;
 //   * C_out <= 128 with K >= 64: weight-stationary tcgen05 engine;
-//   * K = 32 (stem-like 1x1 layer): register-fed warp-level int8 engine;
+//   * other K = 32 layers: register-fed warp-level int8 engine;
 //   * the single-bit mma.sync and CUDA-core engines never win and serve as fallbacks.
 int auto_engine(const ConvProblem &p)
 {
+    if (conv_lop3_pointwise_k32(p)) return BCNN_ENGINE_LOP3;
     if (p.C_out <= 128 && p.K >= 64 && conv_tc_ws_supports(p)) return BCNN_ENGINE_TC_WS;
     if (p.C_out <= 64 && conv_mma_s8_supports(p)) return BCNN_ENGINE_MMA_S8;
     if (conv_tc_i8_supports(p)) return BCNN_ENGINE_TC_I8;

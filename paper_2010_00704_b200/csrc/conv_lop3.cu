@@ -135,10 +135,98 @@ conv_lop3_kernel(const ConvProblem p)
     }
 }
 
+// Pointwise layer with one word of K (1x1, stride 1, no padding, C_in = 32, C_out <= 32): a pixel is one
+// 32-bit word and an output is one XOR + popcount, so a tile engine only adds overhead.  Each thread
+// turns four pixels per step into four output words: per output bit XOR, POPC, subtract and a funnel
+// shift that collects the sign; the popcount pipe is the bound (measured 13 outputs per clock per SM).  K - 2*pc >= thr  <=>  pc <= floor((K - thr) / 2) =: lim, and the sign bit of lim - pc is the
+// complement of the output bit.
+template <bool FUSED>
+__global__ void __launch_bounds__(256)
+conv_k32_kernel(const ConvProblem p)
+{
+    uint32_t w[32];       // uniform across the grid: weight words and popcount limits
+    int lim[32];
+#pragma unroll
+    for (int n = 0; n < 32; ++n) {
+        w[n] = n < p.C_out ? __ldg(p.w + n) : 0u;
+        lim[n] = 0;
+        if (FUSED) {
+            int t = __ldg(p.thr + n);
+            t = t < -64 ? -64 : (t > 64 ? 64 : t);        // beyond +-K the comparison is constant
+            lim[n] = (32 - t) >> 1;                        // floor: arithmetic shift
+        }
+    }
+    const long groups = p.M >> 2;                          // four consecutive pixels per step
+    const long stride = (long)gridDim.x * blockDim.x;
+    const long first = (long)blockIdx.x * blockDim.x + threadIdx.x;
+    const uint4 *x4 = reinterpret_cast<const uint4 *>(p.x);
+
+    auto pixel = [&](uint32_t xv, long m) -> uint32_t {
+        if (FUSED) {
+            uint32_t acc = 0;
+#pragma unroll
+            for (int n = 31; n >= 0; --n) acc = __funnelshift_l((uint32_t)(lim[n] - __popc(xv ^ w[n])), acc, 1);
+            return ~acc;
+        } else {
+            int32_t *dst = static_cast<int32_t *>(p.out) + m * p.C_out;
+            if (p.C_out == 32) {
+#pragma unroll
+                for (int n4 = 0; n4 < 8; ++n4)
+                    *reinterpret_cast<int4 *>(dst + 4 * n4) =
+                        make_int4(32 - 2 * __popc(xv ^ w[4 * n4]), 32 - 2 * __popc(xv ^ w[4 * n4 + 1]),
+                                  32 - 2 * __popc(xv ^ w[4 * n4 + 2]), 32 - 2 * __popc(xv ^ w[4 * n4 + 3]));
+            } else {
+#pragma unroll
+                for (int n = 0; n < 32; ++n)
+                    if (n < p.C_out) dst[n] = 32 - 2 * __popc(xv ^ w[n]);
+            }
+            return 0;
+        }
+    };
+
+    for (long g = first; g < groups; g += stride) {
+        const uint4 xv = __ldg(x4 + g);
+        uint4 o;
+        o.x = pixel(xv.x, 4 * g);
+        o.y = pixel(xv.y, 4 * g + 1);
+        o.z = pixel(xv.z, 4 * g + 2);
+        o.w = pixel(xv.w, 4 * g + 3);
+        if (FUSED) reinterpret_cast<uint4 *>(p.out)[g] = o;
+    }
+    const long m = 4 * groups + first;                     // up to three tail pixels
+    if (m < p.M) {
+        const uint32_t o = pixel(__ldg(p.x + m), m);
+        if (FUSED) static_cast<uint32_t *>(p.out)[m] = o;
+    }
+}
+
+template <bool FUSED>
+int launch_k32(const ConvProblem &p, cudaStream_t stream)
+{
+    int dev = 0, sms = 148, per_sm = 1;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, conv_k32_kernel<FUSED>, 256, 0) != cudaSuccess || per_sm < 1)
+        per_sm = 1;
+    const long groups = ((long)p.M + 3) / 4;
+    long blocks = (groups + 255) / 256;
+    const long wave = (long)sms * per_sm;                 // one resident wave, grid-stride beyond it
+    if (blocks > wave) blocks = wave;
+    conv_k32_kernel<FUSED><<<(unsigned)blocks, 256, 0, stream>>>(p);
+    return cudaGetLastError() == cudaSuccess ? BCNN_OK : BCNN_ERR_CUDA;
+}
+
 }  // namespace
+
+bool conv_lop3_pointwise_k32(const ConvProblem &p)
+{
+    return p.kh * p.kw == 1 && p.stride == 1 && p.pad == 0 && p.C_in == 32 &&
+           (p.thr ? p.C_out == 32 : p.C_out <= 32);
+}
 
 int launch_conv_lop3(const ConvProblem &p, cudaStream_t stream)
 {
+    if (conv_lop3_pointwise_k32(p)) return p.thr ? launch_k32<true>(p, stream) : launch_k32<false>(p, stream);
     dim3 grid((p.M + BM - 1) / BM, (p.C_out + BN - 1) / BN);
     if (grid.y > 65535) return BCNN_ERR_UNSUPPORTED;
     if (p.thr)

@@ -78,6 +78,10 @@ CONV_SHAPES = [
     (1, 40, 40, 256, 256, 3, 3, 2, 1),     # several M and N tiles, K = 2304
     (5, 14, 14, 512, 64, 3, 3, 1, 1),      # K = 4608
     (1, 3, 3, 32, 32, 5, 5, 1, 2),         # kernel larger than the image interior
+    (3, 20, 19, 32, 32, 1, 1, 1, 0),       # pointwise layer with one word of K, M % 4 == 0
+    (1, 21, 27, 32, 32, 1, 1, 1, 0),       # the same with a tail of three pixels
+    (2, 23, 15, 64, 64, 1, 1, 1, 0),       # 1x1 with 64 channels
+    (1, 2, 2, 32, 32, 1, 1, 1, 0),         # a single group of four pixels
 ]
 
 
