@@ -24,23 +24,18 @@
 //   * the implicit-im2col gather uses a per-K-word table (tap, word offset) and a per-row
 //     tap-validity mask instead of divisions; out-of-image taps are zero-filled by cp.async.
 // Every mbarrier wait is bounded and reports through the device error word.
-#include "bcnn_common.cuh"
+#include "tc_common.cuh"
 
 namespace bcnn {
 
 namespace {
 
-constexpr int BM = 128;
-constexpr int ROWB = 128;                 // bytes of one expanded row per stage (= 128 bits of K)
+using namespace tc;
+
 constexpr int EPI_WARPS = 4;
 constexpr int FIRST_PRODUCER_THREAD = 32 * (1 + EPI_WARPS);
 constexpr int PF = 3;                     // packed-word stages in flight per producer thread
 constexpr int MAX_SMEM = 227 * 1024;
-constexpr uint32_t WAIT_LIMIT = 1u << 17;
-// upper bound (ns) for which one try_wait may suspend the thread: waiting warps then leave
-// the issue slots to the warps that have work; the wake-up on phase completion is immediate
-constexpr uint32_t SUSPEND_HINT_NS = 20000;
-constexpr uint32_t SLEEP_NS = 100;
 
 constexpr int ERR_PRODUCER_TIMEOUT = 111;
 constexpr int ERR_MMA_TIMEOUT = 112;
@@ -67,182 +62,6 @@ template <int BN, int G, bool DUAL> struct Cfg {
     static constexpr int BITS_BYTES = PF * PROD_THREADS * 16;
 };
 
-__device__ __forceinline__ uint32_t smem_u32(const void *p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
-
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
-{
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar)
-{
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
-{
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok) : "r"(bar), "r"(parity), "r"(SUSPEND_HINT_NS) : "memory");
-    return ok != 0;
-}
-// Bounded wait with back-off.  A polling warp competes with the MMA-issuing warp for issue
-// slots, so after a first failed poll the waiter sleeps between polls.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *err, int code)
-{
-    if (mbar_try_wait(bar, parity)) return true;
-    for (uint32_t it = 0; it < WAIT_LIMIT; ++it) {
-        __nanosleep(SLEEP_NS);
-        if (mbar_try_wait(bar, parity)) return true;
-        if ((it & 255u) == 255u && *abort_flag) return false;
-    }
-    *abort_flag = 1;
-    if (err) atomicCAS(err, 0, code);
-    return false;
-}
-__device__ __forceinline__ void fence_async_proxy() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_commit(uint32_t bar)
-{
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void tc_mma_i8(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate)
-{
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, {%5, %6, %7, %8}, p;\n\t}"
-        ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate), "r"(0u), "r"(0u), "r"(0u), "r"(0u)
-        : "memory");
-}
-// Predicated forms for the issuer warp: every lane executes the same straight-line code and
-// only the elected lane's predicate is true, so there is no branch to reconverge from.  The
-// descriptors are passed as (low word, high word); only the low word (start address) varies.
-__device__ __forceinline__ void tc_mma_i8_pred(uint32_t d_tmem, uint32_t a_lo, uint32_t b_lo, uint32_t desc_hi,
-                                               uint32_t idesc, uint32_t accumulate, uint32_t pred)
-{
-    asm volatile(
-        "{\n\t.reg .pred p, q;\n\t.reg .b64 da, db;\n\t"
-        "setp.ne.b32 p, %5, 0;\n\t"
-        "setp.ne.b32 q, %6, 0;\n\t"
-        "mov.b64 da, {%1, %3};\n\t"
-        "mov.b64 db, {%2, %3};\n\t"
-        "@q tcgen05.mma.cta_group::1.kind::i8 [%0], da, db, %4, {%7, %7, %7, %7}, p;\n\t}"
-        ::"r"(d_tmem), "r"(a_lo), "r"(b_lo), "r"(desc_hi), "r"(idesc), "r"(accumulate), "r"(pred), "r"(0u)
-        : "memory");
-}
-// A operand from tensor memory (128 lanes x 8 columns = 128 rows x 32 bytes of K), B from shared memory.
-__device__ __forceinline__ void tc_mma_i8_ts_pred(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t desc_hi,
-                                                  uint32_t idesc, uint32_t accumulate, uint32_t pred)
-{
-    asm volatile(
-        "{\n\t.reg .pred p, q;\n\t.reg .b64 db;\n\t"
-        "setp.ne.b32 p, %5, 0;\n\t"
-        "setp.ne.b32 q, %6, 0;\n\t"
-        "mov.b64 db, {%2, %3};\n\t"
-        "@q tcgen05.mma.cta_group::1.kind::i8 [%0], [%1], db, %4, {%7, %7, %7, %7}, p;\n\t}"
-        ::"r"(d_tmem), "r"(a_tmem), "r"(b_lo), "r"(desc_hi), "r"(idesc), "r"(accumulate), "r"(pred), "r"(0u)
-        : "memory");
-}
-// 32 columns of this warp's 32 lanes <- 32 registers; returns once the store has completed.
-__device__ __forceinline__ void tc_st32(uint32_t taddr, const uint32_t (&v)[32])
-{
-    asm volatile(
-        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
-        "{%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,"
-        "%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32};\n\t"
-        "tcgen05.wait::st.sync.aligned;"
-        ::"r"(taddr),
-          "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]),
-          "r"(v[8]), "r"(v[9]), "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15]),
-          "r"(v[16]), "r"(v[17]), "r"(v[18]), "r"(v[19]), "r"(v[20]), "r"(v[21]), "r"(v[22]), "r"(v[23]),
-          "r"(v[24]), "r"(v[25]), "r"(v[26]), "r"(v[27]), "r"(v[28]), "r"(v[29]), "r"(v[30]), "r"(v[31])
-        : "memory");
-}
-__device__ __forceinline__ void tc_commit_pred(uint32_t bar, uint32_t pred)
-{
-    asm volatile(
-        "{\n\t.reg .pred q;\n\tsetp.ne.b32 q, %1, 0;\n\t"
-        "@q tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n\t}"
-        ::"r"(bar), "r"(pred) : "memory");
-}
-
-// 32 accumulator columns of this warp's 32 rows.  The load and its completion wait are one asm
-// statement so that no use of the destination registers can be scheduled between them.
-__device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&v)[32])
-{
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-        "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
-        "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];\n\t"
-        "tcgen05.wait::ld.sync.aligned;"
-        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
-          "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
-          "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
-          "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
-        : "r"(taddr) : "memory");
-}
-__device__ __forceinline__ uint32_t tc_ld1(uint32_t taddr)
-{
-    uint32_t v;
-    asm volatile("tcgen05.ld.sync.aligned.32x32b.x1.b32 {%0}, [%1];\n\ttcgen05.wait::ld.sync.aligned;"
-                 : "=r"(v) : "r"(taddr) : "memory");
-    return v;
-}
-
-// K-major tile, 128-byte rows, 128-byte swizzle, 8-row groups 1024 bytes apart, descriptor version 1.
-__device__ __forceinline__ uint64_t make_desc(uint32_t saddr)
-{
-    const uint32_t lo = ((saddr & 0x3FFFFu) >> 4) | (1u << 16);
-    const uint32_t hi = (1024u >> 4) | (1u << 14) | (2u << 29);
-    return (static_cast<uint64_t>(hi) << 32) | lo;
-}
-// unsigned 8-bit A and B (K-major), int32 accumulate, M = 128, N = n.
-__device__ __forceinline__ constexpr uint32_t make_idesc(int n)
-{
-    return (2u << 4) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
-}
-__device__ __forceinline__ void st_shared_v4(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d)
-{
-    asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
-}
-__device__ __forceinline__ uint4 ld_shared_v4(uint32_t addr)
-{
-    uint4 v;
-    asm volatile("ld.shared.v4.b32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr) : "memory");
-    return v;
-}
-__device__ __forceinline__ void cp_async16(uint32_t dst, const void *src, bool valid)
-{
-    const int n = valid ? 16 : 0;
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(n) : "memory");
-}
-__device__ __forceinline__ void cp_async4(uint32_t dst, const void *src, bool valid)
-{
-    const int n = valid ? 4 : 0;
-    asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;" ::"r"(dst), "l"(src), "r"(n) : "memory");
-}
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
-template <int N>
-__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
-
-__device__ __forceinline__ void expand_store_a(uint32_t w, uint32_t row_addr, int xr, int c)
-{
-    st_shared_v4(row_addr + (uint32_t)(((c) ^ xr) << 4),
-                 w & 0x01010101u, w & 0x02020202u, w & 0x04040404u, w & 0x08080808u);
-    st_shared_v4(row_addr + (uint32_t)(((c + 1) ^ xr) << 4),
-                 w & 0x10101010u, w & 0x20202020u, w & 0x40404040u, w & 0x80808080u);
-}
-__device__ __forceinline__ void expand_store_w(uint32_t w, uint32_t row_addr, int xr, int c)
-{
-    st_shared_v4(row_addr + (uint32_t)(((c) ^ xr) << 4),
-                 (w << 7) & 0x80808080u, (w << 5) & 0x40404040u, (w << 3) & 0x20202020u, (w << 1) & 0x10101010u);
-    st_shared_v4(row_addr + (uint32_t)(((c + 1) ^ xr) << 4),
-                 (w >> 1) & 0x08080808u, (w >> 3) & 0x04040404u, (w >> 5) & 0x02020202u, (w >> 7) & 0x01010101u);
-}
-
 struct WsLayout {
     int ktiles;       // 128-bit K stages
     int smem;         // dynamic shared memory in bytes
@@ -254,7 +73,7 @@ __host__ __device__ inline WsLayout ws_layout(int kwords)
     using C = Cfg<BN, G, DUAL>;
     WsLayout l;
     l.ktiles = (kwords + 3) >> 2;
-    l.smem = 1024 + l.ktiles * C::W_TILE_BYTES + C::BITS_BYTES + BN * 4 + l.ktiles * 4 * 4;
+    l.smem = 1024 + l.ktiles * C::W_TILE_BYTES + C::BITS_BYTES + BN * 4 + l.ktiles * 32;
     // Tensor memory is shared out by the resident CTAs (all 512 columns, or 256 each for two): ask
     // for enough shared memory that no further CTA of this kernel fits on the SM (it would sit in
     // tcgen05.alloc until a neighbour exits).
@@ -290,7 +109,7 @@ conv_tc_ws_kernel(const ConvProblem p)
     const uint32_t wexp = (smem_u32(smem_raw) + 1023u) & ~1023u;          // [ktiles][BNX rows][128 B]
     const uint32_t bits_ring = wexp + (uint32_t)ktiles * C::W_TILE_BYTES; // [PF][PROD_THREADS][16 B]
     const uint32_t colc_addr = bits_ring + C::BITS_BYTES;                 // [BN] int32
-    const uint32_t ktab_addr = colc_addr + BN * 4;                        // [ktiles*4] int32: (word offset << 5) | tap
+    const uint32_t ktab_addr = colc_addr + BN * 4;                        // unit table: [ktiles * 4 / gw] x {word offset, tap bit}
     const uint32_t bar0 = smem_u32(bars);
     auto full_bar = [&](int s) { return bar0 + 8u * s; };
     auto empty_bar = [&](int s) { return bar0 + 8u * (MAX_STAGES + s); };
@@ -342,17 +161,8 @@ conv_tc_ws_kernel(const ConvProblem p)
         const int cst = FUSED ? -32 * ((c < p.C_out ? __ldg(p.thr + c) : 0) - p.K + 2 * pop) : p.K - 2 * pop;
         asm volatile("st.shared.b32 [%0], %1;" ::"r"(colc_addr + 4u * c), "r"(cst) : "memory");
     }
-    for (int kword = tid; kword < ktiles * 4; kword += C::THREADS) {
-        int entry = 0;
-        if (kword < p.kwords) {
-            const int tap = kword / p.cw, cj = kword - tap * p.cw;
-            const int r = tap / p.kw, t = tap - r * p.kw;
-            entry = (((r * p.W + t) * p.cw + cj) << 5) | tap;
-        } else {
-            entry = 31;                      // tap 31 is never valid (at most 31 taps are supported)
-        }
-        asm volatile("st.shared.b32 [%0], %1;" ::"r"(ktab_addr + 4u * kword), "r"(entry) : "memory");
-    }
+    const int gw = gather_width(p.cw);
+    build_unit_table(p, ktab_addr, ktiles * (4 / gw), gw, tid, C::THREADS);
     fence_async_proxy();
     tc_fence_before();
     __syncthreads();
@@ -496,101 +306,80 @@ conv_tc_ws_kernel(const ConvProblem p)
         }
     } else {
         // ------------------------------------------------------------------ producers
+        // Group g takes items g, g + G, ... of the CTA's flattened (tile, stage) list.  Per item a
+        // thread copies its row's 128 bits of K into its staging slot (PF items ahead), then expands
+        // the oldest staged item into the ring slot of tensor memory.
         const int ptid = tid - FIRST_PRODUCER_THREAD;
         const int grp = ptid >> 7;                               // group = 4 consecutive warps
         const int quad = warp & 3;                               // tensor-memory lane quadrant this warp may write
         const int row = quad * 32 + lane;                        // the four warps of a group cover rows 0..127
-        const uint32_t my_bits = bits_ring + (uint32_t)ptid * 16u;
-        const bool a16 = (p.cw & 3) == 0;
-        const bool plain = (p.kh * p.kw == 1 && p.stride == 1 && p.pad == 0);
+        constexpr uint32_t SLOT_BYTES = C::PROD_THREADS * 16u;
+        const uint32_t bits0 = bits_ring + (uint32_t)ptid * 16u, bits_end = bits0 + PF * SLOT_BYTES;
+        const uint32_t st_addr0 = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)C::A_COL0;
+        const uint32_t lane0 = lane == 0 ? 1u : 0u;
+        const TileStep step = make_tile_step(p, (uint32_t)BM * gridDim.x);
 
-        // this thread's items: grp, grp + G, grp + 2G, ... of the CTA's flattened (tile, stage) list
-        // ---- load cursor
-        int l_it = grp, l_ti = 0, l_kt = grp, l_slot = 0;
-        bool l_fresh = true;                 // the row set-up of tile l_ti is still to be done
-        const uint32_t *l_base = p.x;
-        uint32_t l_mask = 0;
-        auto l_locate = [&]() {              // (tile, stage) of l_it; refresh the row when the tile changes
-            while (l_kt >= ktiles) { l_kt -= ktiles; ++l_ti; l_fresh = true; }
-            if (l_fresh) {
-                l_fresh = false;
-                const int m = ((int)blockIdx.x + l_ti * (int)gridDim.x) * BM + row;
-                const bool ok = m < p.M;
-                if (plain) {
-                    l_base = p.x + (long)(ok ? m : 0) * p.cw;
-                    l_mask = ok ? 1u : 0u;
-                } else {
-                    const RowCoord rc = row_coord(p, ok ? m : 0);
-                    l_base = p.x + (((long)rc.b * p.H + rc.ih0) * p.W + rc.iw0) * p.cw;
-                    uint32_t colbits = 0, mask = 0;
-                    for (int t = 0; t < p.kw; ++t)
-                        if (rc.iw0 + t >= 0 && rc.iw0 + t < p.W) colbits |= 1u << t;
-                    for (int r = 0; r < p.kh; ++r)
-                        if (rc.ih0 + r >= 0 && rc.ih0 + r < p.H) mask |= colbits << (r * p.kw);
-                    l_mask = ok ? mask : 0u;
+        auto produce = [&](auto gw_tag) {
+            constexpr int GW = decltype(gw_tag)::value;
+            constexpr uint32_t TAB_STAGE = (4 / GW) * 8u;        // table bytes per stage
+            // ---- load cursor
+            RowCursor rc;
+            rc.m = (uint32_t)blockIdx.x * BM + (uint32_t)row;
+            row_locate(p, rc);
+            int l_kt = grp;
+            int l_left = total_items > grp ? (total_items - grp + G - 1) / G : 0;
+            while (l_kt >= ktiles) { l_kt -= ktiles; row_step(p, step, rc); }
+            row_window(p, step, rc);
+            uint32_t l_dst = bits0;
+            auto issue = [&]() {
+                gather_stage<GW>(p.x, rc, ktab_addr + (uint32_t)l_kt * TAB_STAGE, l_dst);
+                l_dst += SLOT_BYTES;
+                if (l_dst == bits_end) l_dst = bits0;
+                --l_left;
+                l_kt += G;
+                if (l_kt >= ktiles) {
+                    do { l_kt -= ktiles; row_step(p, step, rc); } while (l_kt >= ktiles);
+                    row_window(p, step, rc);
                 }
-            }
-        };
-        auto issue_load = [&]() {
-            l_locate();
-            const uint32_t dst = my_bits + (uint32_t)l_slot * (C::PROD_THREADS * 16u);
-            if (a16) {
-                int entry;
-                asm volatile("ld.shared.b32 %0, [%1];" : "=r"(entry) : "r"(ktab_addr + 16u * l_kt));
-                const bool ok = (l_mask >> (entry & 31)) & 1u;
-                cp_async16(dst, ok ? l_base + (entry >> 5) : p.x, ok);
-            } else {
-                const uint4 e4 = ld_shared_v4(ktab_addr + 16u * l_kt);
-                const int ent[4] = {(int)e4.x, (int)e4.y, (int)e4.z, (int)e4.w};
-#pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    const bool ok = (l_mask >> (ent[e] & 31)) & 1u;
-                    cp_async4(dst + 4u * e, ok ? l_base + (ent[e] >> 5) : p.x, ok);
-                }
-            }
-            l_it += G;
-            l_kt += G;
-            if (++l_slot == PF) l_slot = 0;
-        };
-
-        int issued = 0;                       // groups committed so far
+            };
 #pragma unroll 1
-        for (; issued < PF - 1; ++issued) {
-            if (l_it < total_items) issue_load();
-            cp_async_commit();
-        }
-
-        // ---- expand cursor
-        int c_slot = 0;
-        int s = grp;                          // ring slot of item `it` and its parity, kept incrementally
-        uint32_t phase = 1;                   // first pass through the ring: slots are free
-        while (s >= STAGES) { s -= STAGES; phase ^= 1u; }
-        bool alive = true;
-        for (int it = grp; it < total_items; it += G) {
-            if (l_it < total_items) issue_load();
-            cp_async_commit();
-            cp_async_wait<PF - 1>();
-            const uint4 bits = ld_shared_v4(my_bits + (uint32_t)c_slot * (C::PROD_THREADS * 16u));
-            if (++c_slot == PF) c_slot = 0;
-            alive = mbar_wait(empty_bar(s), phase, abort_flag, p.err, ERR_PRODUCER_TIMEOUT);
-            alive = __all_sync(0xffffffffu, alive);
-            if (!alive) break;
-            tc_fence_after();     // the MMAs that read this slot are complete (their commit released it)
-            // expanded row -> 32 columns of this lane: column 8*e + j = word j of K word e (bytes 0 or 2^j)
-            uint32_t v[32];
-            const uint32_t wds[4] = {bits.x, bits.y, bits.z, bits.w};
+            for (int n = 0; n < PF - 1; ++n) {
+                if (l_left > 0) issue();
+                cp_async_commit();
+            }
+            // ---- expand cursor
+            uint32_t c_src = bits0;
+            int s = grp;                          // ring slot (G <= STAGES) and its parity
+            uint32_t phase = 1;                   // first pass through the ring: slots are free
+#pragma unroll 1
+            for (int it = grp; it < total_items; it += G) {
+                if (l_left > 0) issue();
+                cp_async_commit();
+                cp_async_wait<PF - 1>();
+                const uint4 bits = ld_shared_v4(c_src);
+                c_src += SLOT_BYTES;
+                if (c_src == bits_end) c_src = bits0;
+                if (!mbar_wait_warp(empty_bar(s), phase, abort_flag, p.err, ERR_PRODUCER_TIMEOUT)) break;
+                tc_fence_after();     // the MMAs that read this slot are complete (their commit released it)
+                // expanded row -> 32 columns of this lane: column 8*e + j = word j of K word e (bytes 0 or 2^j)
+                uint32_t v[32];
+                const uint32_t wds[4] = {bits.x, bits.y, bits.z, bits.w};
 #pragma unroll
-            for (int e = 0; e < 4; ++e)
+                for (int e = 0; e < 4; ++e)
 #pragma unroll
-                for (int j = 0; j < 8; ++j) v[8 * e + j] = wds[e] & (0x01010101u << j);
-            tc_st32(tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(C::A_COL0 + s * 32), v);
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(full_bar(s));
-            s += G;
-            while (s >= STAGES) { s -= STAGES; phase ^= 1u; }
-        }
-        cp_async_wait<0>();
+                    for (int j = 0; j < 8; ++j) v[8 * e + j] = wds[e] & (0x01010101u << j);
+                tc_st32(st_addr0 + (uint32_t)s * 32u, v);
+                tc_fence_before();
+                __syncwarp();
+                mbar_arrive_pred(full_bar(s), lane0);
+                s += G;
+                if (s >= STAGES) { s -= STAGES; phase ^= 1u; }
+            }
+            cp_async_wait<0>();
+        };
+        if (gw == 4) produce(IntC<4>{});
+        else if (gw == 2) produce(IntC<2>{});
+        else produce(IntC<1>{});
     }
 
     tc_fence_before();
@@ -633,8 +422,8 @@ bool conv_tc_ws_supports(const ConvProblem &p)
 {
     if (p.thr != nullptr && (p.C_out % 32 != 0)) return false;
     if (p.C_out > 128 || p.kh * p.kw > 31 || p.K > (1 << 16)) return false;
-    // word offsets of the K-word table are shifted left by 5 bits
-    if ((long)(p.kh * (long)p.W + p.kw) * p.cw >= (1L << 26)) return false;
+    // rows address the input by 32-bit word offsets
+    if ((long)p.B * p.H * p.W * p.cw >= (1L << 31)) return false;
     if (p.C_out <= 32) return fits<32, 4, false>(p);
     if (p.C_out <= 64) return fits<64, 4, false>(p);
     return fits<128, 4, false>(p) || fits<128, 2, false>(p);

@@ -35,10 +35,10 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
     return ok != 0;
 }
 // Bounded wait with back-off.  A polling warp competes with the MMA-issuing warp for issue
-// slots, so after a first failed poll the waiter sleeps between polls.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *err, int code)
+// slots, so after a first failed poll the waiter sleeps between polls.  The polling loop is kept
+// out of line: the common case is one successful try_wait.
+static __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *err, int code)
 {
-    if (mbar_try_wait(bar, parity)) return true;
     for (uint32_t it = 0; it < WAIT_LIMIT; ++it) {
         __nanosleep(SLEEP_NS);
         if (mbar_try_wait(bar, parity)) return true;
@@ -47,6 +47,26 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     *abort_flag = 1;
     if (err) atomicCAS(err, 0, code);
     return false;
+}
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *err, int code)
+{
+    if (mbar_try_wait(bar, parity)) return true;
+    return mbar_wait_slow(bar, parity, abort_flag, err, code);
+}
+// Whole-warp wait: one try_wait per lane and a vote in the common case.
+__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *err, int code)
+{
+    bool ok = mbar_try_wait(bar, parity);
+    if (__all_sync(0xffffffffu, ok)) return true;
+    if (!ok) ok = mbar_wait_slow(bar, parity, abort_flag, err, code);
+    return __all_sync(0xffffffffu, ok);
+}
+__device__ __forceinline__ void mbar_arrive_pred(uint32_t bar, uint32_t pred)
+{
+    asm volatile(
+        "{\n\t.reg .pred q;\n\tsetp.ne.b32 q, %1, 0;\n\t"
+        "@q mbarrier.arrive.shared::cta.b64 _, [%0];\n\t}"
+        ::"r"(bar), "r"(pred) : "memory");
 }
 __device__ __forceinline__ void fence_async_proxy() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
@@ -190,6 +210,117 @@ __device__ __forceinline__ void expand_store_w(uint32_t w, uint32_t row_addr, in
                  (w >> 1) & 0x08080808u, (w >> 3) & 0x04040404u, (w >> 5) & 0x02020202u, (w >> 7) & 0x01010101u);
 }
 
+// ---- implicit-im2col gather -----------------------------------------------------------------------
+// K is cut into units of GW words that never straddle a tap: GW = 4 (one 16-byte copy) when a pixel
+// is a multiple of four words, 2 when it is even, else 1.  The unit table holds, per unit, the word
+// offset from the row's top-left input pixel and the tap's bit (0 for the zero padding of K beyond
+// kwords); a row carries the word offset of its top-left input pixel and the mask of its taps that
+// fall inside the image, so one unit costs a mask test, an add and a copy with zero fill.
+__host__ __device__ __forceinline__ int gather_width(int cw) { return (cw & 3) == 0 ? 4 : ((cw & 1) == 0 ? 2 : 1); }
+
+template <int V> struct IntC { static constexpr int value = V; };
+
+__device__ __forceinline__ void build_unit_table(const ConvProblem &p, uint32_t tab_addr, int units, int gw, int tid, int nthreads)
+{
+    for (int u = tid; u < units; u += nthreads) {
+        const int kword = u * gw;
+        uint32_t off = 0, bit = 0;
+        if (kword < p.kwords) {
+            const int tap = kword / p.cw, cj = kword - tap * p.cw;
+            const int r = tap / p.kw, t = tap - r * p.kw;
+            off = (uint32_t)((r * p.W + t) * p.cw + cj);
+            bit = 1u << tap;
+        }
+        asm volatile("st.shared.v2.b32 [%0], {%1,%2};" ::"r"(tab_addr + 8u * u), "r"(off), "r"(bit) : "memory");
+    }
+}
+
+// Advance of a CTA from one of its row tiles to the next: a constant number of rows, split once into
+// whole images, output rows and output columns, so that a row's coordinates follow by carries.
+struct TileStep {
+    uint32_t rows;
+    int db, doh, dow;
+    uint32_t pat;            // bit r*kw for every kernel row r
+};
+__device__ __forceinline__ TileStep make_tile_step(const ConvProblem &p, uint32_t rows)
+{
+    TileStep s;
+    const uint32_t ohw = (uint32_t)(p.OH * p.OW);
+    s.rows = rows;
+    s.db = (int)(rows / ohw);
+    const uint32_t rem = rows - (uint32_t)s.db * ohw;
+    s.doh = (int)(rem / (uint32_t)p.OW);
+    s.dow = (int)(rem - (uint32_t)s.doh * (uint32_t)p.OW);
+    s.pat = 0;
+    for (int r = 0; r < p.kh; ++r) s.pat |= 1u << (r * p.kw);
+    return s;
+}
+struct RowCursor {
+    uint32_t m;              // row of the implicit patch matrix
+    int b, oh, ow;
+    int base;                // word offset of the top-left input pixel (may be negative)
+    uint32_t mask;           // taps inside the image; 0 for rows beyond M
+};
+__device__ __forceinline__ void row_locate(const ConvProblem &p, RowCursor &rc)
+{
+    const uint32_t ohw = (uint32_t)(p.OH * p.OW);
+    rc.b = (int)exact_div(rc.m, p.ohw_mul, p.ohw_shift);
+    const uint32_t rem = rc.m - (uint32_t)rc.b * ohw;
+    rc.oh = (int)exact_div(rem, p.ow_mul, p.ow_shift);
+    rc.ow = (int)(rem - (uint32_t)rc.oh * (uint32_t)p.OW);
+}
+__device__ __forceinline__ void row_step(const ConvProblem &p, const TileStep &s, RowCursor &rc)
+{
+    rc.m += s.rows;
+    rc.ow += s.dow;
+    if (rc.ow >= p.OW) { rc.ow -= p.OW; ++rc.oh; }
+    rc.oh += s.doh;
+    if (rc.oh >= p.OH) { rc.oh -= p.OH; ++rc.b; }
+    rc.b += s.db;
+}
+__device__ __forceinline__ uint32_t low_bits(int n) { return (1u << n) - 1u; }   // 0 <= n <= 31
+__device__ __forceinline__ void row_window(const ConvProblem &p, const TileStep &s, RowCursor &rc)
+{
+    const int ih0 = rc.oh * p.stride - p.pad, iw0 = rc.ow * p.stride - p.pad;
+    rc.base = ((rc.b * p.H + ih0) * p.W + iw0) * p.cw;
+    // taps t with 0 <= iw0 + t < W and r with 0 <= ih0 + r < H (an empty range gives an empty mask)
+    const int clo = min(max(-iw0, 0), p.kw), chi = max(min(p.W - iw0, p.kw), 0);
+    const int rlo = min(max(-ih0, 0), p.kh), rhi = max(min(p.H - ih0, p.kh), 0);
+    const uint32_t cols = low_bits(chi) & ~low_bits(clo);
+    const uint32_t rows = s.pat & low_bits(rhi * p.kw) & ~low_bits(rlo * p.kw);
+    rc.mask = rc.m < (uint32_t)p.M ? cols * rows : 0u;
+}
+template <int BYTES>
+__device__ __forceinline__ void cp_async_zfill(uint32_t dst, const void *src, uint32_t nbytes)
+{
+    if (BYTES == 16)
+        asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(nbytes) : "memory");
+    else if (BYTES == 8)
+        asm volatile("cp.async.ca.shared.global [%0], [%1], 8, %2;" ::"r"(dst), "l"(src), "r"(nbytes) : "memory");
+    else
+        asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;" ::"r"(dst), "l"(src), "r"(nbytes) : "memory");
+}
+// One 128-bit stage (4 / GW units, table entries at `tab`) of the row `rc` -> 16 bytes at `dst`.
+template <int GW>
+__device__ __forceinline__ void gather_stage(const uint32_t *x, const RowCursor &rc, uint32_t tab, uint32_t dst)
+{
+    constexpr int U = 4 / GW;
+    uint32_t ent[2 * U];
+    if (U == 1) {
+        asm volatile("ld.shared.v2.b32 {%0,%1}, [%2];" : "=r"(ent[0]), "=r"(ent[1]) : "r"(tab));
+    } else {
+#pragma unroll
+        for (int h = 0; h < U / 2; ++h)
+            asm volatile("ld.shared.v4.b32 {%0,%1,%2,%3}, [%4];"
+                         : "=r"(ent[4 * h]), "=r"(ent[4 * h + 1]), "=r"(ent[4 * h + 2]), "=r"(ent[4 * h + 3]) : "r"(tab + 16u * h));
+    }
+#pragma unroll
+    for (int u = 0; u < U; ++u) {
+        const bool ok = (rc.mask & ent[2 * u + 1]) != 0u;
+        const int idx = ok ? rc.base + (int)ent[2 * u] : 0;
+        cp_async_zfill<GW * 4>(dst + (uint32_t)(u * GW * 4), x + idx, ok ? (uint32_t)(GW * 4) : 0u);
+    }
+}
 
 }  // namespace tc
 }  // namespace bcnn
