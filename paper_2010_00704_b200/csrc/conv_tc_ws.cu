@@ -45,14 +45,18 @@ constexpr int ERR_EPILOGUE_TIMEOUT = 113;
 template <int BN, int G, bool DUAL> struct Cfg {
     static constexpr int BNX = BN + 16;                       // + the all-ones row (MMA N is a multiple of 16)
     static constexpr int PROD_THREADS = G * BM;
-    static constexpr int CONTROL_WARP = (FIRST_PRODUCER_THREAD + PROD_THREADS) / 32;   // last warp
-    static constexpr int THREADS = FIRST_PRODUCER_THREAD + PROD_THREADS + 32;
     // Tensor memory (512 columns): NBUF accumulator buffers of BNX columns, then the activation ring,
     // one stage = 128 rows x 128 expanded bytes = 32 columns.
     static constexpr int TMEM_COLS = DUAL ? 256 : 512;
     static constexpr int NBUF = DUAL ? (BN == 128 ? 1 : 2) : (BN == 32 ? 4 : (BN == 64 ? 3 : 2));
+    static constexpr int NISS = NBUF >= 2 ? 2 : 1;            // MMA issuer warps; they take the CTA's tiles in turn
+    static constexpr int CONTROL_WARP = (FIRST_PRODUCER_THREAD + PROD_THREADS) / 32;
+    static constexpr int ISSUER2_WARP = CONTROL_WARP + 1;     // second MMA issuer (odd tiles), when there are two buffers
+    static constexpr int THREADS = FIRST_PRODUCER_THREAD + PROD_THREADS + 32 + (NISS - 1) * 32;
     static constexpr int A_COL0 = NBUF * BNX;
-    static constexpr int STAGES = (TMEM_COLS - A_COL0) / 32 > 8 ? 8 : (TMEM_COLS - A_COL0) / 32;
+    // named barriers 1 .. NISS * MAX_RING release the stages to the issuers: one id per (issuer, slot)
+    static constexpr int MAX_RING = NISS == 2 ? 7 : 8;
+    static constexpr int STAGES = (TMEM_COLS - A_COL0) / 32 > MAX_RING ? MAX_RING : (TMEM_COLS - A_COL0) / 32;
     static constexpr int CTAS_PER_SM = DUAL ? 2 : 1;
     // registers are granted in blocks of 8 per thread: bound the pair of CTAs to 64 registers per thread
     static constexpr int BOUND_THREADS = DUAL ? 512 : THREADS;
@@ -169,47 +173,55 @@ conv_tc_ws_kernel(const ConvProblem p)
     tc_fence_after();
     const uint32_t tmem_base = tmem_base_smem;
 
-    if (warp == 0) {
-        // ------------------------------------------------------------------ MMA issuer
-        // This warp never touches memory: a load or an mbarrier wait issued after tensor-core
+    if (warp == 0 || (C::NISS == 2 && warp == C::ISSUER2_WARP)) {
+        // ------------------------------------------------------------------ MMA issuers
+        // These warps never touch memory: a load or an mbarrier wait issued after tensor-core
         // instructions holds the issuing thread until they have drained (measured: +230 cycles per
         // stage), a named barrier does not.  The control warp does the waiting and releases one
-        // stage at a time through named barrier 1 + slot.
+        // stage at a time through a named barrier per (issuer, slot).  Issuing costs more than the MMAs take
+        // (the warp shares its scheduler with producer warps), so with two accumulator buffers two
+        // issuers take the CTA's tiles in turn: all MMAs of a tile come from one thread, in order,
+        // and the next tile's are issued beside them as soon as its stages are in the ring.
         constexpr uint32_t idesc = make_idesc(BNX);
         const uint64_t desc0 = make_desc(0);
         const uint32_t desc_hi = (uint32_t)(desc0 >> 32);
         const uint32_t a_tmem0 = tmem_base + (uint32_t)C::A_COL0;                // + slot * 32 columns
         const uint32_t b_lo0 = (uint32_t)desc0 | ((wexp & 0x3FFFFu) >> 4);       // + kt * (W_TILE_BYTES / 16)
         const uint32_t elected = lane == 0 ? 1u : 0u;
-        int s = 0, buf = 0;
-        for (int ti = 0; ti < my_tiles; ++ti) {
+        const int me = warp == 0 ? 0 : 1;
+        const int skip = (C::NISS - 1) * ktiles % STAGES;                        // slots of the other issuer's tile
+        int s = me * ktiles % STAGES, buf = me % NBUF;
+        for (int ti = me; ti < my_tiles; ti += C::NISS) {
             const uint32_t d_tmem = tmem_base + (uint32_t)(buf * BNX);
             const uint32_t tfull = tfull_bar(buf);
             for (int kt = 0; kt < ktiles; ++kt) {
                 const uint32_t a_t = a_tmem0 + (uint32_t)s * 32u;
                 const uint32_t b_lo = b_lo0 + (uint32_t)kt * (C::W_TILE_BYTES >> 4);
                 const int nk = p.kwords - 4 * kt;                 // 32 bits of K per instruction; skip the zero tail
-                const uint32_t e1 = nk > 1 ? elected : 0u, e2 = nk > 2 ? elected : 0u, e3 = nk > 3 ? elected : 0u;
-                const uint32_t last = (kt == ktiles - 1) ? elected : 0u;
                 const uint32_t ebar = empty_bar(s);
-                asm volatile("bar.sync %0, 64;" ::"r"(1 + s) : "memory");
+                asm volatile("bar.sync %0, 64;" ::"r"(1 + me * C::MAX_RING + s) : "memory");
                 tc_fence_after();
                 // per 32 bytes of K: 8 tensor-memory columns of A, +2 (16-byte units) in the B descriptor
+                // (warp-uniform branches: an instruction whose predicate is off in every lane still costs its issue time)
                 tc_mma_i8_ts_pred(d_tmem, a_t, b_lo, desc_hi, idesc, kt > 0 ? 1u : 0u, elected);
-                tc_mma_i8_ts_pred(d_tmem, a_t + 8u, b_lo + 2u, desc_hi, idesc, 1u, e1);
-                tc_mma_i8_ts_pred(d_tmem, a_t + 16u, b_lo + 4u, desc_hi, idesc, 1u, e2);
-                tc_mma_i8_ts_pred(d_tmem, a_t + 24u, b_lo + 6u, desc_hi, idesc, 1u, e3);
+                if (nk > 1) tc_mma_i8_ts_pred(d_tmem, a_t + 8u, b_lo + 2u, desc_hi, idesc, 1u, elected);
+                if (nk > 2) tc_mma_i8_ts_pred(d_tmem, a_t + 16u, b_lo + 4u, desc_hi, idesc, 1u, elected);
+                if (nk > 3) tc_mma_i8_ts_pred(d_tmem, a_t + 24u, b_lo + 6u, desc_hi, idesc, 1u, elected);
                 tc_commit_pred(ebar, elected);
-                tc_commit_pred(tfull, last);
+                if (kt == ktiles - 1) tc_commit_pred(tfull, elected);
                 if (++s == STAGES) s = 0;
             }
-            if (++buf == NBUF) buf = 0;
+            s += skip;
+            if (s >= STAGES) s -= STAGES;
+            buf += C::NISS;
+            while (buf >= NBUF) buf -= NBUF;
         }
     } else if (warp == C::CONTROL_WARP) {
         // ------------------------------------------------------------------ control: waits for the issuer
-        // Stage `it` is released (bar.arrive on 1 + slot) once its ring slot is full and, for a tile's
-        // first stage, once the accumulator buffer is free.  The slot being full implies that the
-        // issuer is past the previous use of the same named barrier (it committed that slot's release).
+        // A stage is released to the issuer that owns its tile (bar.arrive on that issuer's barrier of
+        // the slot) once its ring slot is full and, for a tile's first stage, once the accumulator
+        // buffer is free.  The slot being full implies that every earlier use of the slot has been
+        // committed, so the owner is past the previous use of the same named barrier.
         // After a time-out the remaining stages are released without waiting so that the issuer,
         // whose barrier wait has no time limit, always terminates; the error word tells the host.
         int s = 0, buf = 0;
@@ -220,7 +232,7 @@ conv_tc_ws_kernel(const ConvProblem p)
             for (int kt = 0; kt < ktiles; ++kt) {
                 if (lane == 0 && alive) alive = mbar_wait(full_bar(s), ring_phase, abort_flag, p.err, ERR_MMA_TIMEOUT);
                 __syncwarp();
-                asm volatile("bar.arrive %0, 64;" ::"r"(1 + s) : "memory");
+                asm volatile("bar.arrive %0, 64;" ::"r"(1 + (ti % C::NISS) * C::MAX_RING + s) : "memory");
                 if (++s == STAGES) { s = 0; ring_phase ^= 1u; }
             }
             if (++buf == NBUF) { buf = 0; buf_phase ^= 1u; }
