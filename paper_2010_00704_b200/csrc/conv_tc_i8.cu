@@ -89,7 +89,7 @@ conv_tc_i8_kernel(const ConvProblem p, const int ktab_words)
     const uint32_t wring = (smem_u32(smem_raw) + 1023u) & ~1023u;         // [STAGES][BN rows][128 B]
     const uint32_t bits_ring = wring + STAGES * C::W_BYTES;               // [PF][PROD_THREADS][16 B]
     const uint32_t consts = bits_ring + C::BITS_BYTES;                    // [SLOTS][G][BM + BN] int32
-    const uint32_t ktab_addr = consts + C::CONST_BYTES;                   // [ktab_words] (word offset << 5) | tap
+    const uint32_t ktab_addr = consts + C::CONST_BYTES;                   // unit table of the gather: {word offset, tap bit}
     const uint32_t bar0 = smem_u32(bars);
     auto full_bar = [&](int s) { return bar0 + 8u * s; };
     auto empty_bar = [&](int s) { return bar0 + 8u * (8 + s); };
@@ -113,15 +113,8 @@ conv_tc_i8_kernel(const ConvProblem p, const int ktab_words)
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_smem)), "r"(512u) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
-    for (int kword = tid; kword < ktab_words; kword += C::THREADS) {
-        int entry = 31;                          // tap 31 is never valid (at most 31 taps)
-        if (kword < p.kwords) {
-            const int tap = kword / p.cw, cj = kword - tap * p.cw;
-            const int r = tap / p.kw, t = tap - r * p.kw;
-            entry = (((r * p.W + t) * p.cw + cj) << 5) | tap;
-        }
-        asm volatile("st.shared.b32 [%0], %1;" ::"r"(ktab_addr + 4u * kword), "r"(entry) : "memory");
-    }
+    const int gwidth = gather_width(p.cw);
+    build_unit_table(p, ktab_addr, ktiles * (4 / gwidth), gwidth, tid, C::THREADS);
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
@@ -143,18 +136,17 @@ conv_tc_i8_kernel(const ConvProblem p, const int ktab_words)
                 const uint32_t a_t = a_tmem0 + (uint32_t)s * 32u;
                 const uint32_t b_lo = b_lo0 + (uint32_t)s * (C::W_BYTES >> 4);
                 const int nk = p.kwords - 4 * kt;                 // 32 bits of K per instruction; skip the zero tail
-                const uint32_t e1 = nk > 1 ? elected : 0u, e2 = nk > 2 ? elected : 0u, e3 = nk > 3 ? elected : 0u;
-                const uint32_t last = (kt == ktiles - 1) ? elected : 0u;
                 const uint32_t ebar = empty_bar(s);
                 asm volatile("bar.sync %0, 64;" ::"r"(1 + s) : "memory");
                 tc_fence_after();
                 // per 32 bytes of K: 8 tensor-memory columns of A, +2 (16-byte units) in the B descriptor
                 tc_mma_i8_ts_pred(d_tmem, a_t, b_lo, desc_hi, idesc, kt > 0 ? 1u : 0u, elected);
-                tc_mma_i8_ts_pred(d_tmem, a_t + 8u, b_lo + 2u, desc_hi, idesc, 1u, e1);
-                tc_mma_i8_ts_pred(d_tmem, a_t + 16u, b_lo + 4u, desc_hi, idesc, 1u, e2);
-                tc_mma_i8_ts_pred(d_tmem, a_t + 24u, b_lo + 6u, desc_hi, idesc, 1u, e3);
+                // (warp-uniform branches: an instruction whose predicate is off in every lane still costs its issue time)
+                if (nk > 1) tc_mma_i8_ts_pred(d_tmem, a_t + 8u, b_lo + 2u, desc_hi, idesc, 1u, elected);
+                if (nk > 2) tc_mma_i8_ts_pred(d_tmem, a_t + 16u, b_lo + 4u, desc_hi, idesc, 1u, elected);
+                if (nk > 3) tc_mma_i8_ts_pred(d_tmem, a_t + 24u, b_lo + 6u, desc_hi, idesc, 1u, elected);
                 tc_commit_pred(ebar, elected);
-                tc_commit_pred(tfull, last);
+                if (kt == ktiles - 1) tc_commit_pred(tfull, elected);
                 if (++s == STAGES) s = 0;
             }
             if (++buf == NBUF) buf = 0;
@@ -282,112 +274,103 @@ conv_tc_i8_kernel(const ConvProblem p, const int ktab_words)
     } else {
         // ------------------------------------------------------------------ producers
         const int pw = warp - C::FIRST_PRODUCER_WARP;            // producer warp index
-        const int grp = pw / C::GROUP_WARPS, gw = pw - grp * C::GROUP_WARPS;
-        const bool is_a = gw < 4;
+        const int grp = pw / C::GROUP_WARPS, wi = pw - grp * C::GROUP_WARPS;
+        const bool is_a = wi < 4;
         // activation warps are matched to tensor-memory lane quadrants (a warp may only touch
         // lanes 32 * (warp % 4) ...): the first four warps of a group have four distinct residues
         const int quad = warp & 3;
-        const int row = is_a ? quad * 32 + lane : (gw - 4) * 32 + lane;   // row of the A or of the W tile
+        const int row = is_a ? quad * 32 + lane : (wi - 4) * 32 + lane;   // row of the A or of the W tile
         const int ptid = tid - 32 * C::FIRST_PRODUCER_WARP;
         const int crow = is_a ? row : BM + row;                  // index into a constants part
-        const uint32_t my_bits = bits_ring + (uint32_t)ptid * 16u;
-        const bool a16 = (p.cw & 3) == 0;
+        constexpr uint32_t SLOT_BYTES = C::PROD_THREADS * 16u;
+        const uint32_t bits0 = bits_ring + (uint32_t)ptid * 16u, bits_end = bits0 + PF * SLOT_BYTES;
+        const uint32_t st_addr0 = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)C::A_COL0;
+        const uint32_t lane0 = lane == 0 ? 1u : 0u;
         const bool w16 = (p.kwords & 3) == 0;
-        const bool plain = (p.kh * p.kw == 1 && p.stride == 1 && p.pad == 0);
+        const TileStep step = make_tile_step(p, (uint32_t)BM * gridDim.x);
 
         // this thread's items: grp, grp + G, ... of the CTA's flattened (tile, stage) list
-        // ---- load cursor
-        int l_it = grp, l_ti = 0, l_kt = grp, l_slot = 0;
-        bool l_fresh = true;
-        const uint32_t *l_base = p.x;
-        uint32_t l_mask = 0;
-        auto l_locate = [&]() {
-            while (l_kt >= ktiles) { l_kt -= ktiles; ++l_ti; l_fresh = true; }
-            if (l_fresh) {
-                l_fresh = false;
-                const int tile = (int)blockIdx.x + l_ti * (int)gridDim.x;
-                const int n_tile = tile / m_tiles, m_tile = tile - n_tile * m_tiles;
+        // ---- load cursor: tile (n_tile, m_tile) and, per role, the activation row or the weight row
+        int l_kt = grp;
+        int l_left = total_items > grp ? (total_items - grp + G - 1) / G : 0;
+        int l_n = (int)blockIdx.x / m_tiles, l_m = (int)blockIdx.x - l_n * m_tiles;
+        RowCursor rc;
+        rc.m = (uint32_t)l_m * BM + (uint32_t)row;
+        rc.base = 0;
+        rc.mask = 0;
+        const uint32_t *wrow = p.w;
+        bool wok = false;
+        if (is_a) row_locate(p, rc);
+        auto next_tile = [&]() {             // the CTA's next tile: gridDim.x further along (n_tile, m_tile)
+            l_m += (int)gridDim.x;
+            if (l_m < m_tiles) {
+                if (is_a) row_step(p, step, rc);
+            } else {
+                do { l_m -= m_tiles; ++l_n; } while (l_m >= m_tiles);
                 if (is_a) {
-                    const int m = m_tile * BM + row;
-                    const bool ok = m < p.M;
-                    if (plain) {
-                        l_base = p.x + (long)(ok ? m : 0) * p.cw;
-                        l_mask = ok ? 1u : 0u;
-                    } else {
-                        const RowCoord rc = row_coord(p, ok ? m : 0);
-                        l_base = p.x + (((long)rc.b * p.H + rc.ih0) * p.W + rc.iw0) * p.cw;
-                        uint32_t colbits = 0, mask = 0;
-                        for (int t = 0; t < p.kw; ++t)
-                            if (rc.iw0 + t >= 0 && rc.iw0 + t < p.W) colbits |= 1u << t;
-                        for (int r = 0; r < p.kh; ++r)
-                            if (rc.ih0 + r >= 0 && rc.ih0 + r < p.H) mask |= colbits << (r * p.kw);
-                        l_mask = ok ? mask : 0u;
-                    }
-                } else {
-                    const int n = n_tile * BN + row;
-                    const bool ok = n < p.C_out;
-                    l_base = p.w + (long)(ok ? n : 0) * p.kwords;
-                    l_mask = ok ? 1u : 0u;
+                    rc.m = (uint32_t)l_m * BM + (uint32_t)row;
+                    row_locate(p, rc);
                 }
             }
         };
-        auto issue_load = [&]() {
-            l_locate();
-            const uint32_t dst = my_bits + (uint32_t)l_slot * (C::PROD_THREADS * 16u);
-            if (!is_a || plain) {
-                // contiguous K: word kt*4 + e of the row
-                const bool rok = l_mask != 0;
-                if (is_a ? a16 : w16) {
-                    cp_async16(dst, rok ? l_base + l_kt * 4 : p.x, rok);
-                } else {
-#pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        const int kword = l_kt * 4 + e;
-                        const bool ok = rok && kword < p.kwords;
-                        cp_async4(dst + 4u * e, ok ? l_base + kword : p.x, ok);
-                    }
-                }
-            } else if (a16) {
-                int entry;
-                asm volatile("ld.shared.b32 %0, [%1];" : "=r"(entry) : "r"(ktab_addr + 16u * l_kt));
-                const bool ok = (l_mask >> (entry & 31)) & 1u;
-                cp_async16(dst, ok ? l_base + (entry >> 5) : p.x, ok);
+        auto tile_ready = [&]() {            // per-tile values of the row after the cursor moved
+            if (is_a) {
+                row_window(p, step, rc);
             } else {
-                const uint4 e4 = ld_shared_v4(ktab_addr + 16u * l_kt);
-                const int ent[4] = {(int)e4.x, (int)e4.y, (int)e4.z, (int)e4.w};
+                const int n = l_n * BN + row;
+                wok = n < p.C_out;
+                wrow = p.w + (long)(wok ? n : 0) * p.kwords;
+            }
+        };
+        while (l_kt >= ktiles) { l_kt -= ktiles; next_tile(); }
+        tile_ready();
+        uint32_t l_dst = bits0;
+        auto issue_load = [&]() {
+            if (is_a) {
+                if (gwidth == 4) gather_stage<4>(p.x, rc, ktab_addr + (uint32_t)l_kt * 8u, l_dst);
+                else if (gwidth == 2) gather_stage<2>(p.x, rc, ktab_addr + (uint32_t)l_kt * 16u, l_dst);
+                else gather_stage<1>(p.x, rc, ktab_addr + (uint32_t)l_kt * 32u, l_dst);
+            } else if (w16) {
+                cp_async_zfill<16>(l_dst, wok ? wrow + l_kt * 4 : p.w, wok ? 16u : 0u);
+            } else {
 #pragma unroll
                 for (int e = 0; e < 4; ++e) {
-                    const bool ok = (l_mask >> (ent[e] & 31)) & 1u;
-                    cp_async4(dst + 4u * e, ok ? l_base + (ent[e] >> 5) : p.x, ok);
+                    const int kword = l_kt * 4 + e;
+                    const bool ok = wok && kword < p.kwords;
+                    cp_async_zfill<4>(l_dst + 4u * e, ok ? wrow + kword : p.w, ok ? 4u : 0u);
                 }
             }
-            l_it += G;
+            l_dst += SLOT_BYTES;
+            if (l_dst == bits_end) l_dst = bits0;
+            --l_left;
             l_kt += G;
-            if (++l_slot == PF) l_slot = 0;
+            if (l_kt >= ktiles) {
+                do { l_kt -= ktiles; next_tile(); } while (l_kt >= ktiles);
+                tile_ready();
+            }
         };
 
 #pragma unroll 1
         for (int i = 0; i < PF - 1; ++i) {
-            if (l_it < total_items) issue_load();
+            if (l_left > 0) issue_load();
             cp_async_commit();
         }
 
         // ---- expand cursor
-        int c_slot = 0, c_ti = 0, c_kt = grp, pop = 0;
-        int s = grp;
+        uint32_t c_src = bits0;
+        int c_ti = 0, c_kt = grp, pop = 0;
+        int s = grp;                          // ring slot (G <= STAGES) and its parity
         uint32_t phase = 1;                   // first pass through the ring: slots are free
-        while (s >= STAGES) { s -= STAGES; phase ^= 1u; }
-        bool alive = true;
+#pragma unroll 1
         for (int it = grp; it < total_items; it += G) {
-            if (l_it < total_items) issue_load();
+            if (l_left > 0) issue_load();
             cp_async_commit();
             cp_async_wait<PF - 1>();
-            const uint4 bits = ld_shared_v4(my_bits + (uint32_t)c_slot * (C::PROD_THREADS * 16u));
-            if (++c_slot == PF) c_slot = 0;
+            const uint4 bits = ld_shared_v4(c_src);
+            c_src += SLOT_BYTES;
+            if (c_src == bits_end) c_src = bits0;
             while (c_kt >= ktiles) { c_kt -= ktiles; ++c_ti; }
-            alive = mbar_wait(empty_bar(s), phase, abort_flag, p.err, ERR_PRODUCER_TIMEOUT);
-            alive = __all_sync(0xffffffffu, alive);
-            if (!alive) break;
+            if (!mbar_wait_warp(empty_bar(s), phase, abort_flag, p.err, ERR_PRODUCER_TIMEOUT)) break;
             pop += __popc(bits.x) + __popc(bits.y) + __popc(bits.z) + __popc(bits.w);
             if (c_kt + G >= ktiles) {
                 // this group's last stage of the tile: leave its partial constants for the epilogue.
@@ -414,7 +397,7 @@ conv_tc_i8_kernel(const ConvProblem p, const int ktab_words)
                 for (int e = 0; e < 4; ++e)
 #pragma unroll
                     for (int j = 0; j < 8; ++j) v[8 * e + j] = wds[e] & (0x01010101u << j);
-                tc_st32(tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(C::A_COL0 + s * 32), v);
+                tc_st32(st_addr0 + (uint32_t)s * 32u, v);
                 tc_fence_before();
             } else {
                 const uint32_t row_addr = wring + (uint32_t)s * C::W_BYTES + (uint32_t)row * ROWB;
@@ -426,9 +409,9 @@ conv_tc_i8_kernel(const ConvProblem p, const int ktab_words)
                 fence_async_proxy();  // generic-proxy stores -> visible to the MMA (async proxy)
             }
             __syncwarp();
-            if (lane == 0) mbar_arrive(full_bar(s));
+            mbar_arrive_pred(full_bar(s), lane0);
             s += G;
-            while (s >= STAGES) { s -= STAGES; phase ^= 1u; }
+            if (s >= STAGES) { s -= STAGES; phase ^= 1u; }
             c_kt += G;
         }
         cp_async_wait<0>();
@@ -443,8 +426,7 @@ conv_tc_i8_kernel(const ConvProblem p, const int ktab_words)
 
 int ktab_words_for(const ConvProblem &p)
 {
-    const bool plain = (p.kh * p.kw == 1 && p.stride == 1 && p.pad == 0);
-    return plain ? 0 : ((p.kwords + 3) & ~3);
+    return ((p.kwords + 3) >> 2) * 8;        // at most four units of two words per 128-bit stage
 }
 
 template <int BN>
@@ -474,7 +456,7 @@ bool conv_tc_i8_supports(const ConvProblem &p)
 {
     if (p.thr != nullptr && (p.C_out % 32 != 0)) return false;
     if (p.kh * p.kw > 31) return false;                       // one validity bit per tap
-    if ((long)(p.kh * (long)p.W + p.kw) * p.cw >= (1L << 26)) return false;   // table offsets are shifted by 5 bits
+    if ((long)p.B * p.H * p.W * p.cw >= (1L << 31)) return false;     // rows address the input by 32-bit word offsets
     if (smem_bytes<256>(ktab_words_for(p)) > MAX_SMEM) return false;   // the K-word table of the gather must fit
     // the epilogue constants (about 3K << 5) must stay below 2^31
     return p.K <= (1 << 20);

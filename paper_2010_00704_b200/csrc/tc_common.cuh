@@ -202,12 +202,15 @@ __device__ __forceinline__ void expand_store_a(uint32_t w, uint32_t row_addr, in
     st_shared_v4(row_addr + (uint32_t)(((c + 1) ^ xr) << 4),
                  w & 0x10101010u, w & 0x20202020u, w & 0x40404040u, w & 0x80808080u);
 }
+// Weights take the value 2^(7-j) where the activation byte is 2^j: reverse the bits of each byte once
+// (bit j+8i -> bit (7-j)+8i), after which every output word is again a single AND.
 __device__ __forceinline__ void expand_store_w(uint32_t w, uint32_t row_addr, int xr, int c)
 {
+    const uint32_t r = __byte_perm(__brev(w), 0u, 0x0123u);
     st_shared_v4(row_addr + (uint32_t)(((c) ^ xr) << 4),
-                 (w << 7) & 0x80808080u, (w << 5) & 0x40404040u, (w << 3) & 0x20202020u, (w << 1) & 0x10101010u);
+                 r & 0x80808080u, r & 0x40404040u, r & 0x20202020u, r & 0x10101010u);
     st_shared_v4(row_addr + (uint32_t)(((c + 1) ^ xr) << 4),
-                 (w >> 1) & 0x08080808u, (w >> 3) & 0x04040404u, (w >> 5) & 0x02020202u, (w >> 7) & 0x01010101u);
+                 r & 0x08080808u, r & 0x04040404u, r & 0x02020202u, r & 0x01010101u);
 }
 
 // ---- implicit-im2col gather -----------------------------------------------------------------------
