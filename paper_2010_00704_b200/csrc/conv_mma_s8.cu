@@ -255,7 +255,8 @@ int launch_na(const ConvProblem &p, cudaStream_t stream)
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     const long nblocks = ((long)p.M + 16 * MA - 1) / (16 * MA);
     void (*k)(const ConvProblem) = p.thr ? conv_mma_s8_kernel<NA, true> : conv_mma_s8_kernel<NA, false>;
-    if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return BCNN_ERR_CUDA;
+    // a property of the kernel, not of the launch: always the limit, so that captured launches stay valid
+    if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM) != cudaSuccess) return BCNN_ERR_CUDA;
     int per_sm = 1;
     if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k, THREADS, smem) != cudaSuccess || per_sm < 1) per_sm = 1;
     // persistent grid: every resident CTA slot of the chip, split over the N tiles

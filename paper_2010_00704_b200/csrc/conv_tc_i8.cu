@@ -445,7 +445,9 @@ int launch_bn(const ConvProblem &p0, cudaStream_t stream)
     const int ktw = ktab_words_for(p);
     const int smem = smem_bytes<BN>(ktw);
     void (*k)(const ConvProblem, const int) = p.thr ? conv_tc_i8_kernel<BN, true> : conv_tc_i8_kernel<BN, false>;
-    if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return BCNN_ERR_CUDA;
+    // the attribute is a property of the kernel, not of the launch: always the limit, so that a captured
+    // launch stays valid whatever later calls with other shapes ask for
+    if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM) != cudaSuccess) return BCNN_ERR_CUDA;
     k<<<grid, Cfg<BN>::THREADS, smem, stream>>>(p, ktw);
     return cudaGetLastError() == cudaSuccess ? BCNN_OK : BCNN_ERR_CUDA;
 }

@@ -415,7 +415,9 @@ int launch_ws(const ConvProblem &p0, cudaStream_t stream)
     const long slots = (long)sms * C::CTAS_PER_SM;
     const unsigned grid = (unsigned)(m_tiles < slots ? m_tiles : slots);
     void (*k)(const ConvProblem) = p.thr ? conv_tc_ws_kernel<BN, G, DUAL, true> : conv_tc_ws_kernel<BN, G, DUAL, false>;
-    if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, L.smem) != cudaSuccess) return BCNN_ERR_CUDA;
+    // the attribute is a property of the kernel, not of the launch: always the configuration's limit, so
+    // that a captured launch stays valid whatever later calls with other shapes ask for
+    if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, DUAL ? 113 * 1024 : MAX_SMEM - 1024) != cudaSuccess) return BCNN_ERR_CUDA;
     k<<<grid, C::THREADS, L.smem, stream>>>(p);
     return cudaGetLastError() == cudaSuccess ? BCNN_OK : BCNN_ERR_CUDA;
 }
@@ -425,7 +427,7 @@ int launch_ws(const ConvProblem &p0, cudaStream_t stream)
 template <int BN, int G, bool DUAL>
 bool fits(const ConvProblem &p)
 {
-    return ws_layout<BN, G, DUAL>(p.kwords).smem + 512 <= (DUAL ? 113 * 1024 : MAX_SMEM);
+    return ws_layout<BN, G, DUAL>(p.kwords).smem <= (DUAL ? 113 * 1024 : MAX_SMEM - 1024);
 }
 
 }  // namespace
