@@ -49,14 +49,10 @@ template <int BN, int G, bool DUAL> struct Cfg {
     // one stage = 128 rows x 128 expanded bytes = 32 columns.
     static constexpr int TMEM_COLS = DUAL ? 256 : 512;
     static constexpr int NBUF = DUAL ? (BN == 128 ? 1 : 2) : (BN == 32 ? 4 : (BN == 64 ? 3 : 2));
-    static constexpr int NISS = NBUF >= 2 ? 2 : 1;            // MMA issuer warps; they take the CTA's tiles in turn
     static constexpr int CONTROL_WARP = (FIRST_PRODUCER_THREAD + PROD_THREADS) / 32;
-    static constexpr int ISSUER2_WARP = CONTROL_WARP + 1;     // second MMA issuer (odd tiles), when there are two buffers
-    static constexpr int THREADS = FIRST_PRODUCER_THREAD + PROD_THREADS + 32 + (NISS - 1) * 32;
+    static constexpr int THREADS = FIRST_PRODUCER_THREAD + PROD_THREADS + 32;
     static constexpr int A_COL0 = NBUF * BNX;
-    // named barriers 1 .. NISS * MAX_RING release the stages to the issuers: one id per (issuer, slot)
-    static constexpr int MAX_RING = NISS == 2 ? 7 : 8;
-    static constexpr int STAGES = (TMEM_COLS - A_COL0) / 32 > MAX_RING ? MAX_RING : (TMEM_COLS - A_COL0) / 32;
+    static constexpr int STAGES = (TMEM_COLS - A_COL0) / 32 > 8 ? 8 : (TMEM_COLS - A_COL0) / 32;
     static constexpr int CTAS_PER_SM = DUAL ? 2 : 1;
     // registers are granted in blocks of 8 per thread: bound the pair of CTAs to 64 registers per thread
     static constexpr int BOUND_THREADS = DUAL ? 512 : THREADS;
@@ -68,6 +64,8 @@ template <int BN, int G, bool DUAL> struct Cfg {
 
 struct WsLayout {
     int ktiles;       // 128-bit K stages
+    int row_kt;       // > 0: producers work tile by tile (all row_kt stages of a row at once), see the producers
+    int bits_bytes;   // staging ring of the packed words
     int smem;         // dynamic shared memory in bytes
 };
 
@@ -77,7 +75,13 @@ __host__ __device__ inline WsLayout ws_layout(int kwords)
     using C = Cfg<BN, G, DUAL>;
     WsLayout l;
     l.ktiles = (kwords + 3) >> 2;
-    l.smem = 1024 + l.ktiles * C::W_TILE_BYTES + C::BITS_BYTES + BN * 4 + l.ktiles * 32;
+    // Short K: a producer group takes whole tiles in turn instead of single stages, so the per-tile work
+    // (row coordinates, tap mask, bookkeeping) is done once per row and tile.  A group then runs up to
+    // (G - 1) * ktiles + 1 ring slots ahead of the slot it waits for; the parity waits need the ring
+    // to be at least that deep.
+    l.row_kt = (l.ktiles <= 3 && C::STAGES >= (G - 1) * l.ktiles + 1) ? l.ktiles : 0;
+    l.bits_bytes = C::BITS_BYTES * (l.row_kt ? l.row_kt : 1);
+    l.smem = 1024 + l.ktiles * C::W_TILE_BYTES + l.bits_bytes + BN * 4 + l.ktiles * 32;
     // Tensor memory is shared out by the resident CTAs (all 512 columns, or 256 each for two): ask
     // for enough shared memory that no further CTA of this kernel fits on the SM (it would sit in
     // tcgen05.alloc until a neighbour exits).
@@ -112,7 +116,7 @@ conv_tc_ws_kernel(const ConvProblem p)
     // shared-memory map (all 1024-byte aligned where the MMA reads)
     const uint32_t wexp = (smem_u32(smem_raw) + 1023u) & ~1023u;          // [ktiles][BNX rows][128 B]
     const uint32_t bits_ring = wexp + (uint32_t)ktiles * C::W_TILE_BYTES; // [PF][PROD_THREADS][16 B]
-    const uint32_t colc_addr = bits_ring + C::BITS_BYTES;                 // [BN] int32
+    const uint32_t colc_addr = bits_ring + (uint32_t)L.bits_bytes;                 // [BN] int32
     const uint32_t ktab_addr = colc_addr + BN * 4;                        // unit table: [ktiles * 4 / gw] x {word offset, tap bit}
     const uint32_t bar0 = smem_u32(bars);
     auto full_bar = [&](int s) { return bar0 + 8u * s; };
@@ -173,25 +177,22 @@ conv_tc_ws_kernel(const ConvProblem p)
     tc_fence_after();
     const uint32_t tmem_base = tmem_base_smem;
 
-    if (warp == 0 || (C::NISS == 2 && warp == C::ISSUER2_WARP)) {
-        // ------------------------------------------------------------------ MMA issuers
-        // These warps never touch memory: a load or an mbarrier wait issued after tensor-core
+    if (warp == 0) {
+        // ------------------------------------------------------------------ MMA issuer
+        // This warp never touches memory: a load or an mbarrier wait issued after tensor-core
         // instructions holds the issuing thread until they have drained (measured: +230 cycles per
         // stage), a named barrier does not.  The control warp does the waiting and releases one
-        // stage at a time through a named barrier per (issuer, slot).  Issuing costs more than the MMAs take
-        // (the warp shares its scheduler with producer warps), so with two accumulator buffers two
-        // issuers take the CTA's tiles in turn: all MMAs of a tile come from one thread, in order,
-        // and the next tile's are issued beside them as soon as its stages are in the ring.
+        // stage at a time through named barrier 1 + slot.  There is one issuer on purpose: the
+        // producers' parity waits rely on the ring being consumed in order (a second issuer working on
+        // the next tile lets a late slot fall two phases behind a waiting producer).
         constexpr uint32_t idesc = make_idesc(BNX);
         const uint64_t desc0 = make_desc(0);
         const uint32_t desc_hi = (uint32_t)(desc0 >> 32);
         const uint32_t a_tmem0 = tmem_base + (uint32_t)C::A_COL0;                // + slot * 32 columns
         const uint32_t b_lo0 = (uint32_t)desc0 | ((wexp & 0x3FFFFu) >> 4);       // + kt * (W_TILE_BYTES / 16)
         const uint32_t elected = lane == 0 ? 1u : 0u;
-        const int me = warp == 0 ? 0 : 1;
-        const int skip = (C::NISS - 1) * ktiles % STAGES;                        // slots of the other issuer's tile
-        int s = me * ktiles % STAGES, buf = me % NBUF;
-        for (int ti = me; ti < my_tiles; ti += C::NISS) {
+        int s = 0, buf = 0;
+        for (int ti = 0; ti < my_tiles; ++ti) {
             const uint32_t d_tmem = tmem_base + (uint32_t)(buf * BNX);
             const uint32_t tfull = tfull_bar(buf);
             for (int kt = 0; kt < ktiles; ++kt) {
@@ -199,7 +200,7 @@ conv_tc_ws_kernel(const ConvProblem p)
                 const uint32_t b_lo = b_lo0 + (uint32_t)kt * (C::W_TILE_BYTES >> 4);
                 const int nk = p.kwords - 4 * kt;                 // 32 bits of K per instruction; skip the zero tail
                 const uint32_t ebar = empty_bar(s);
-                asm volatile("bar.sync %0, 64;" ::"r"(1 + me * C::MAX_RING + s) : "memory");
+                asm volatile("bar.sync %0, 64;" ::"r"(1 + s) : "memory");
                 tc_fence_after();
                 // per 32 bytes of K: 8 tensor-memory columns of A, +2 (16-byte units) in the B descriptor
                 // (warp-uniform branches: an instruction whose predicate is off in every lane still costs its issue time)
@@ -211,17 +212,13 @@ conv_tc_ws_kernel(const ConvProblem p)
                 if (kt == ktiles - 1) tc_commit_pred(tfull, elected);
                 if (++s == STAGES) s = 0;
             }
-            s += skip;
-            if (s >= STAGES) s -= STAGES;
-            buf += C::NISS;
-            while (buf >= NBUF) buf -= NBUF;
+            if (++buf == NBUF) buf = 0;
         }
     } else if (warp == C::CONTROL_WARP) {
         // ------------------------------------------------------------------ control: waits for the issuer
-        // A stage is released to the issuer that owns its tile (bar.arrive on that issuer's barrier of
-        // the slot) once its ring slot is full and, for a tile's first stage, once the accumulator
-        // buffer is free.  The slot being full implies that every earlier use of the slot has been
-        // committed, so the owner is past the previous use of the same named barrier.
+        // Stage `it` is released (bar.arrive on 1 + slot) once its ring slot is full and, for a tile's
+        // first stage, once the accumulator buffer is free.  The slot being full implies that the
+        // issuer is past the previous use of the same named barrier (it committed that slot's release).
         // After a time-out the remaining stages are released without waiting so that the issuer,
         // whose barrier wait has no time limit, always terminates; the error word tells the host.
         int s = 0, buf = 0;
@@ -232,7 +229,7 @@ conv_tc_ws_kernel(const ConvProblem p)
             for (int kt = 0; kt < ktiles; ++kt) {
                 if (lane == 0 && alive) alive = mbar_wait(full_bar(s), ring_phase, abort_flag, p.err, ERR_MMA_TIMEOUT);
                 __syncwarp();
-                asm volatile("bar.arrive %0, 64;" ::"r"(1 + (ti % C::NISS) * C::MAX_RING + s) : "memory");
+                asm volatile("bar.arrive %0, 64;" ::"r"(1 + s) : "memory");
                 if (++s == STAGES) { s = 0; ring_phase ^= 1u; }
             }
             if (++buf == NBUF) { buf = 0; buf_phase ^= 1u; }
@@ -389,7 +386,83 @@ conv_tc_ws_kernel(const ConvProblem p)
             }
             cp_async_wait<0>();
         };
-        if (gw == 4) produce(IntC<4>{});
+        // ---- short K: this group's items are the tiles grp, grp + G, ...; all stages of a row are staged
+        // together (PF tiles ahead) and expanded one ring slot after the other
+        auto produce_rows = [&](auto gw_tag, auto kt_tag) {
+            constexpr int GW = decltype(gw_tag)::value;
+            constexpr int KT = decltype(kt_tag)::value;
+            constexpr uint32_t TAB_STAGE = (4 / GW) * 8u;
+            constexpr uint32_t TSLOT_BYTES = SLOT_BYTES * KT;     // one staged tile: [KT][PROD_THREADS][16 B]
+            const uint32_t tend = bits0 + PF * TSLOT_BYTES;
+            const TileStep gstep = make_tile_step(p, (uint32_t)BM * gridDim.x * G);
+            RowCursor rc;
+            rc.m = ((uint32_t)blockIdx.x + (uint32_t)grp * gridDim.x) * BM + (uint32_t)row;
+            row_locate(p, rc);
+            row_window(p, gstep, rc);
+            int l_left = my_tiles > grp ? (my_tiles - grp + G - 1) / G : 0;
+            uint32_t l_dst = bits0;
+            auto issue = [&]() {
+#pragma unroll
+                for (int kt = 0; kt < KT; ++kt)
+                    gather_stage<GW>(p.x, rc, ktab_addr + (uint32_t)kt * TAB_STAGE, l_dst + (uint32_t)kt * SLOT_BYTES);
+                l_dst += TSLOT_BYTES;
+                if (l_dst == tend) l_dst = bits0;
+                --l_left;
+                row_step(p, gstep, rc);
+                row_window(p, gstep, rc);
+            };
+#pragma unroll 1
+            for (int n = 0; n < PF - 1; ++n) {
+                if (l_left > 0) issue();
+                cp_async_commit();
+            }
+            uint32_t c_src = bits0;
+            int s = grp * KT;                     // ring slot of the tile's first stage and its parity
+            uint32_t phase = 1;
+            while (s >= STAGES) { s -= STAGES; phase ^= 1u; }
+#pragma unroll 1
+            for (int ti = grp; ti < my_tiles; ti += G) {
+                if (l_left > 0) issue();
+                cp_async_commit();
+                cp_async_wait<PF - 1>();
+                bool alive = true;
+#pragma unroll
+                for (int kt = 0; kt < KT; ++kt) {
+                    const uint4 bits = ld_shared_v4(c_src + (uint32_t)kt * SLOT_BYTES);
+                    if (alive && !mbar_wait_warp(empty_bar(s), phase, abort_flag, p.err, ERR_PRODUCER_TIMEOUT)) alive = false;
+                    if (alive) {
+                        tc_fence_after();
+                        uint32_t v[32];
+                        const uint32_t wds[4] = {bits.x, bits.y, bits.z, bits.w};
+#pragma unroll
+                        for (int e = 0; e < 4; ++e)
+#pragma unroll
+                            for (int j = 0; j < 8; ++j) v[8 * e + j] = wds[e] & (0x01010101u << j);
+                        tc_st32(st_addr0 + (uint32_t)s * 32u, v);
+                        tc_fence_before();
+                        __syncwarp();
+                        mbar_arrive_pred(full_bar(s), lane0);
+                    }
+                    if (++s == STAGES) { s = 0; phase ^= 1u; }
+                }
+                if (!alive) break;
+                c_src += TSLOT_BYTES;
+                if (c_src == tend) c_src = bits0;
+                s += (G - 1) * KT;                // the other groups' tiles
+                while (s >= STAGES) { s -= STAGES; phase ^= 1u; }
+            }
+            cp_async_wait<0>();
+        };
+        auto rows_by_kt = [&](auto gw_tag) {
+            if (L.row_kt == 1) produce_rows(gw_tag, IntC<1>{});
+            else if (L.row_kt == 2) produce_rows(gw_tag, IntC<2>{});
+            else produce_rows(gw_tag, IntC<3>{});
+        };
+        if (L.row_kt) {
+            if (gw == 4) rows_by_kt(IntC<4>{});
+            else if (gw == 2) rows_by_kt(IntC<2>{});
+            else rows_by_kt(IntC<1>{});
+        } else if (gw == 4) produce(IntC<4>{});
         else if (gw == 2) produce(IntC<2>{});
         else produce(IntC<1>{});
     }
