@@ -46,13 +46,17 @@ class FusedChain:
             pong = torch.empty(max(sizes[1::2]) if len(sizes) > 1 else 16, dtype=torch.uint8, device=self.device)
             self.outs = [(ping if i % 2 == 0 else pong)[:s] for i, s in enumerate(sizes)]
         self.graph = None
+        self.layers_graph = None
         self.launches_per_run = len(self.layers) + (1 if real_input_shape is not None else 0)
 
-    def enqueue(self):
+    def enqueue_pack(self, x_real):
+        H, W, C = self.real_input_shape
+        binding.bcnn_pack(x_real, self.bias, self.in_bits, self.batch, H, W, C, self.replicate)
+
+    def enqueue(self, include_pack: bool = True):
         """Enqueue the whole sequence on the current stream; returns the last layer's packed output."""
-        if self.x_real is not None:
-            H, W, C = self.real_input_shape
-            binding.bcnn_pack(self.x_real, self.bias, self.in_bits, self.batch, H, W, C, self.replicate)
+        if self.x_real is not None and include_pack:
+            self.enqueue_pack(self.x_real)
         cur = self.in_bits
         for l, w, t, o in zip(self.layers, self.w, self.thr, self.outs):
             binding.bcnn_conv2d_b1_fused(cur, w, t, o, self.batch, l.H, l.W, l.C_in, l.C_out, l.k, l.k,
@@ -72,7 +76,43 @@ class FusedChain:
         with torch.cuda.graph(g):
             self.enqueue()
         self.graph = g
+        if self.x_real is not None:
+            # the layers alone, for the host-input pipeline below (its pack stage alternates input buffers)
+            gl = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(gl):
+                self.enqueue(include_pack=False)
+            self.layers_graph = gl
         return g
+
+    def run_from_host(self, x_host: torch.Tensor, out_host: torch.Tensor):
+        """One step from a pinned fp32 host tensor to a pinned host copy of the last layer's packed output.
+
+        Double-buffered: the host-to-device copy of this call's input runs on a copy stream and overlaps
+        the kernels of the previous call (which read the other input buffer).  Everything is enqueued
+        asynchronously; synchronise the device before reading ``out_host``."""
+        if not hasattr(self, "_pipe"):
+            self._pipe = {"stream": torch.cuda.Stream(), "bufs": [self.x_real, torch.empty_like(self.x_real)],
+                          "copied": [torch.cuda.Event(), torch.cuda.Event()],
+                          "consumed": [torch.cuda.Event(), torch.cuda.Event()], "n": 0}
+            for ev in self._pipe["consumed"]:
+                ev.record()
+        pp = self._pipe
+        b = pp["n"] & 1
+        pp["n"] += 1
+        main = torch.cuda.current_stream()
+        with torch.cuda.stream(pp["stream"]):
+            pp["stream"].wait_event(pp["consumed"][b])      # the pack that last read this buffer is done
+            pp["bufs"][b].copy_(x_host, non_blocking=True)
+            pp["copied"][b].record()
+        main.wait_event(pp["copied"][b])
+        self.enqueue_pack(pp["bufs"][b])
+        pp["consumed"][b].record()
+        if getattr(self, "layers_graph", None) is not None:
+            self.layers_graph.replay()
+        else:
+            self.enqueue(include_pack=False)
+        out_host.copy_(self.outs[-1], non_blocking=True)
+        return out_host
 
     def run(self):
         if self.graph is not None:

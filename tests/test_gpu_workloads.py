@@ -147,3 +147,30 @@ def test_backbone18_with_pack_stage_and_graph(bk, oracle):
         cur = oracle.threshold(oracle.conv2d(cur, synth.unpack_bits(w), l.stride, l.pad), t)
     assert np.array_equal(got[:b], cur)
     assert bk.bcnn_device_error() == 0
+
+
+def test_backbone18_from_host_pipeline(bk, oracle):
+    # the host-input entry of the chain: three different inputs in a row through the double-buffered
+    # copy stream; every result must be the one of its own input (checked against the oracle)
+    from paper_2010_00704_b200.chain import FusedChain
+    B = 4
+    layers = wl.BACKBONE18
+    H, W, C, R = wl.BACKBONE18_INPUT
+    rng = synth.rng_for(5, 1234)
+    bias = synth.real_input(rng, (C * R,))
+    _, ws, ts = _chain_inputs(5, layers, 1)
+    ch = FusedChain(layers, B, ws, ts, real_input_shape=(H, W, C), bias=bias, replicate=R)
+    ch.capture()
+    xs = [synth.real_input(rng, (B, H, W, C)) for _ in range(3)]
+    x_hosts = [torch.from_numpy(x.reshape(-1)).pin_memory() for x in xs]
+    out_hosts = [torch.empty(ch.outs[-1].numel(), dtype=torch.uint8).pin_memory() for _ in xs]
+    for xh, oh in zip(x_hosts, out_hosts):
+        ch.run_from_host(xh, oh)
+    torch.cuda.synchronize()
+    for x, oh in zip(xs, out_hosts):
+        cur = oracle.binarize(x[:1], bias, R)
+        for l, w, t in zip(layers, ws, ts):
+            cur = oracle.threshold(oracle.conv2d(cur, synth.unpack_bits(w), l.stride, l.pad), t)
+        got = synth.unpack_bits(oh.numpy().reshape(B, 7, 7, 512 // 8))
+        assert np.array_equal(got[:1], cur)
+    assert bk.bcnn_device_error() == 0
