@@ -315,7 +315,7 @@ def run_gpu(args):
         g_ms = float(sum(per_ms[i + 1] for i in idx))
         g_ops = float(sum(layers[i].ops(B) for i in idx))
         # the CUDA-core kernel sits on the population-count unit: its peak is the xor + popc rate that
-        # tools/engine_peaks measures register-resident (385 TOP/s at 1965 MHz, profiles/engine_bakeoff.md)
+        # tools/engine_peaks measures register-resident (385 TOP/s at 1965 MHz)
         g_bound, g_peak = ("alu", POPC_PEAK_TOPS) if en == "lop3" else ("tensor", tensor_peak)
         groups.append({"kernel": kernel_of[en], "launches_per_step": len(idx), "ms_per_step": g_ms,
                        "share_of_step": g_ms / float(per_ms.sum()), "bound": g_bound,

@@ -69,7 +69,7 @@ int make_conv_problem(ConvProblem &p, const void *x, const void *w, const int32_
     return BCNN_OK;
 }
 
-// Measured on B200 (bench.py --mode sweep, profiles/engine_bakeoff.md):
+// Measured on B200 (bench.py --mode sweep):
 //   * C_out >= 256, or weights too large to keep expanded in shared memory: streaming tcgen05 engine;
 //   * 1x1 layer with C_in = 32 and C_out <= 32 (one XOR + popcount per output): CUDA-core pointwise kernel;
 //   * C_out <= 128 with K >= 64: weight-stationary tcgen05 engine;
