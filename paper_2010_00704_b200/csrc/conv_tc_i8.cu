@@ -126,11 +126,11 @@ conv_tc_i8_kernel(const ConvProblem p, const int ktab_words)
         const uint64_t desc0 = make_desc(0);
         const uint32_t desc_hi = (uint32_t)(desc0 >> 32);
         const uint32_t b_lo0 = (uint32_t)desc0 | ((wring & 0x3FFFFu) >> 4);      // + slot * (W_BYTES / 16)
-        const uint32_t a_tmem0 = tmem_base + (uint32_t)C::A_COL0;                // + slot * 32 columns
-        const uint32_t elected = lane == 0 ? 1u : 0u;
+        const uint32_t tmem_u = __shfl_sync(0xffffffffu, tmem_base, 0);             // warp-uniform copy for the issuer
+        const uint32_t a_tmem0 = tmem_u + (uint32_t)C::A_COL0;                   // + slot * 32 columns
         int s = 0, buf = 0;
         for (int ti = 0; ti < my_tiles; ++ti) {
-            const uint32_t d_tmem = tmem_base + (uint32_t)(buf * BN);
+            const uint32_t d_tmem = tmem_u + (uint32_t)(buf * BN);
             const uint32_t tfull = tfull_bar(buf);
             for (int kt = 0; kt < ktiles; ++kt) {
                 const uint32_t a_t = a_tmem0 + (uint32_t)s * 32u;
@@ -140,13 +140,15 @@ conv_tc_i8_kernel(const ConvProblem p, const int ktab_words)
                 asm volatile("bar.sync %0, 64;" ::"r"(1 + s) : "memory");
                 tc_fence_after();
                 // per 32 bytes of K: 8 tensor-memory columns of A, +2 (16-byte units) in the B descriptor
-                tc_mma_i8_ts_pred(d_tmem, a_t, b_lo, desc_hi, idesc, kt > 0 ? 1u : 0u, elected);
-                // (warp-uniform branches: an instruction whose predicate is off in every lane still costs its issue time)
-                if (nk > 1) tc_mma_i8_ts_pred(d_tmem, a_t + 8u, b_lo + 2u, desc_hi, idesc, 1u, elected);
-                if (nk > 2) tc_mma_i8_ts_pred(d_tmem, a_t + 16u, b_lo + 4u, desc_hi, idesc, 1u, elected);
-                if (nk > 3) tc_mma_i8_ts_pred(d_tmem, a_t + 24u, b_lo + 6u, desc_hi, idesc, 1u, elected);
-                tc_commit_pred(ebar, elected);
-                if (kt == ktiles - 1) tc_commit_pred(tfull, elected);
+                if (elect_one()) {
+                    tc_mma_i8_ts(d_tmem, a_t, b_lo, desc_hi, idesc, kt > 0 ? 1u : 0u);
+                    if (nk > 1) tc_mma_i8_ts(d_tmem, a_t + 8u, b_lo + 2u, desc_hi, idesc, 1u);
+                    if (nk > 2) tc_mma_i8_ts(d_tmem, a_t + 16u, b_lo + 4u, desc_hi, idesc, 1u);
+                    if (nk > 3) tc_mma_i8_ts(d_tmem, a_t + 24u, b_lo + 6u, desc_hi, idesc, 1u);
+                    tc_commit(ebar);
+                    if (kt == ktiles - 1) tc_commit(tfull);
+                }
+                __syncwarp();
                 if (++s == STAGES) s = 0;
             }
             if (++buf == NBUF) buf = 0;
