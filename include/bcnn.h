@@ -115,6 +115,22 @@ int bcnn_conv2d_b1_fused(const void *x_bits, const void *w_bits, const int32_t *
                          int kh, int kw, int stride, int pad, void *stream);
 
 /*
+ * Fused stem: bcnn_pack followed by the first binary 1x1 convolution with its threshold epilogue, without
+ * writing the packed sign tensor in between (Section 4.1: the stem uses the same block, so even the first
+ * convolution is binary; Table 1 "stem replicate": 4 real channels replicated 8x to 32 sign channels;
+ * Section 4.2.1: bias + sign, binary 1x1 convolution, batch norm + next sign folded into a threshold):
+ *   s bit[b][h][w][c]  = (x[b][h][w][c mod C_in] + bias[c] >= 0),                c in [0, R*C_in)
+ *   y bit[b][h][w][co] = (sum_c s[b][h][w][c] * w[co][c] >= thr[co])             s, w in {-1,+1}
+ * The result is bit-identical to the two separate calls.
+ *   x device fp32 NHWC [B][H][W][C_in];  bias device fp32 [R*C_in] or NULL;
+ *   w_bits device, packed [C_out][R*C_in];  thr device int32 [C_out];  y_bits device, packed NHWC [B][H][W][C_out]
+ * Supported shape: C_in = 4, R = 8, C_out = 32 (the paper's stem); anything else returns BCNN_ERR_UNSUPPORTED
+ * and the caller issues the two calls.
+ */
+int bcnn_stem_fused(const float *x, const float *bias, const void *w_bits, const int32_t *thr, void *y_bits,
+                    int B, int H, int W, int C_in, int R, int C_out, void *stream);
+
+/*
  * The same four products with the inner-product engine chosen by the caller (used to
  * compare engines; BCNN_ENGINE_AUTO behaves like the calls above).  thr == NULL selects
  * the int32 output (`out` is int32), otherwise the packed output.  Returns

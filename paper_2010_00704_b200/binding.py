@@ -20,7 +20,7 @@ ENGINES = {"auto": ENGINE_AUTO, "lop3": ENGINE_LOP3, "mma_b1": ENGINE_MMA_B1, "t
            "mma_s8": ENGINE_MMA_S8, "tc_ws": ENGINE_TC_WS}
 
 EXPORTS = (
-    "bcnn_pack", "bcnn_gemm_b1", "bcnn_gemm_b1_fused", "bcnn_conv2d_b1", "bcnn_conv2d_b1_fused",
+    "bcnn_pack", "bcnn_stem_fused", "bcnn_gemm_b1", "bcnn_gemm_b1_fused", "bcnn_conv2d_b1", "bcnn_conv2d_b1_fused",
     "bcnn_conv2d_b1_engine", "bcnn_gemm_b1_engine", "bcnn_auto_engine", "bcnn_device_error", "bcnn_status_string",
     "bcnn_version",
 )
@@ -43,6 +43,7 @@ def load() -> ctypes.CDLL:
         lib = ctypes.CDLL(LIB_PATH)
         vp, i32, i64 = ctypes.c_void_p, ctypes.c_int, ctypes.c_int64
         lib.bcnn_pack.argtypes = [vp, vp, vp, i32, i32, i32, i32, i32, vp]
+        lib.bcnn_stem_fused.argtypes = [vp, vp, vp, vp, vp, i32, i32, i32, i32, i32, i32, vp]
         lib.bcnn_gemm_b1.argtypes = [vp, vp, vp, i64, i32, i32, vp]
         lib.bcnn_gemm_b1_fused.argtypes = [vp, vp, vp, vp, i64, i32, i32, vp]
         lib.bcnn_conv2d_b1.argtypes = [vp, vp, vp] + [i32] * 9 + [vp]
@@ -89,6 +90,15 @@ def bcnn_pack(x: torch.Tensor, bias, out_bits: torch.Tensor, B, H, W, C_in, R=1)
     """x fp32 NHWC device tensor -> packed sign bits written into ``out_bits``."""
     _check(load().bcnn_pack(_p(x), _p(bias), _p(out_bits), B, H, W, C_in, R, _stream()), "bcnn_pack")
     return out_bits
+
+
+def bcnn_stem_fused(x, bias, w_bits, thr, y_bits, B, H, W, C_in, R, C_out):
+    """fp32 NHWC input -> (bias, sign, replication) -> binary 1x1 convolution -> threshold -> packed bits."""
+    if thr is None:
+        raise BcnnError(-1, "bcnn_stem_fused")
+    _check(load().bcnn_stem_fused(_p(x), _p(bias), _p(w_bits), _p(thr), _p(y_bits), B, H, W, C_in, R, C_out,
+                                  _stream()), "bcnn_stem_fused")
+    return y_bits
 
 
 def bcnn_gemm_b1(A_bits, W_bits, C, M, N, K, engine=ENGINE_AUTO):

@@ -2,7 +2,8 @@
 
 Holds the packed weights, thresholds and the ping-pong activation buffers on the device
 and enqueues, through the C ABI, one ``bcnn_pack`` followed by one
-``bcnn_conv2d_b1_fused`` per layer.  It contains no arithmetic of its own.  The launch
+``bcnn_conv2d_b1_fused`` per layer (``bcnn_stem_fused`` replaces the pack and the first layer when the
+shapes are the stem's: 4 real channels x 8 replicas, 1x1 to 32 channels).  It contains no arithmetic of its own.  The launch
 sequence can be captured once into a CUDA graph and replayed.
 """
 from __future__ import annotations
@@ -17,11 +18,13 @@ from .workloads import ConvLayer
 class FusedChain:
     def __init__(self, layers, batch: int, w_bits_list, thr_list, real_input_shape=None, bias=None,
                  replicate: int = 1, engine: int = binding.ENGINE_AUTO, keep_all: bool = False,
-                 device="cuda"):
+                 device="cuda", fuse_stem=None):
         """layers: sequence of ConvLayer; w_bits_list[i]: uint8 numpy [C_out, k, k, C_in/8];
         thr_list[i]: int32 numpy [C_out].  real_input_shape = (H, W, C_real) enables the pack
         stage (fp32 NHWC input, optional per-channel bias, replication factor).
-        keep_all keeps one output buffer per layer (for checking) instead of two ping-pong buffers."""
+        keep_all keeps one output buffer per layer (for checking) instead of two ping-pong buffers.
+        fuse_stem: run pack + first layer as one ``bcnn_stem_fused`` call (the packed input is then never
+        written); default: whenever the shapes allow it and keep_all is off."""
         self.layers = list(layers)
         self.batch = int(batch)
         self.engine = engine
@@ -47,18 +50,31 @@ class FusedChain:
             self.outs = [(ping if i % 2 == 0 else pong)[:s] for i, s in enumerate(sizes)]
         self.graph = None
         self.layers_graph = None
-        self.launches_per_run = len(self.layers) + (1 if real_input_shape is not None else 0)
+        can_fuse = (real_input_shape is not None and real_input_shape[2] == 4 and replicate == 8
+                    and (l0.k, l0.stride, l0.pad, l0.C_in, l0.C_out) == (1, 1, 0, 32, 32)
+                    and engine == binding.ENGINE_AUTO)
+        self.fuse_stem = (can_fuse and not keep_all) if fuse_stem is None else bool(fuse_stem)
+        if self.fuse_stem and not can_fuse:
+            raise ValueError("fuse_stem needs a 4-channel real input replicated 8x and a first 1x1 layer 32 -> 32")
+        self.launches_per_run = len(self.layers) + (1 if real_input_shape is not None and not self.fuse_stem else 0)
 
     def enqueue_pack(self, x_real):
         H, W, C = self.real_input_shape
-        binding.bcnn_pack(x_real, self.bias, self.in_bits, self.batch, H, W, C, self.replicate)
+        if self.fuse_stem:
+            binding.bcnn_stem_fused(x_real, self.bias, self.w[0], self.thr[0], self.outs[0], self.batch, H, W, C,
+                                    self.replicate, self.layers[0].C_out)
+        else:
+            binding.bcnn_pack(x_real, self.bias, self.in_bits, self.batch, H, W, C, self.replicate)
 
     def enqueue(self, include_pack: bool = True):
         """Enqueue the whole sequence on the current stream; returns the last layer's packed output."""
         if self.x_real is not None and include_pack:
             self.enqueue_pack(self.x_real)
         cur = self.in_bits
-        for l, w, t, o in zip(self.layers, self.w, self.thr, self.outs):
+        for i, (l, w, t, o) in enumerate(zip(self.layers, self.w, self.thr, self.outs)):
+            if i == 0 and self.fuse_stem:        # done by enqueue_pack
+                cur = o
+                continue
             binding.bcnn_conv2d_b1_fused(cur, w, t, o, self.batch, l.H, l.W, l.C_in, l.C_out, l.k, l.k,
                                          l.stride, l.pad, engine=self.engine)
             cur = o

@@ -135,6 +135,20 @@ int bcnn_pack(const float *x, const float *bias, void *out_bits,
                        static_cast<cudaStream_t>(stream));
 }
 
+int bcnn_stem_fused(const float *x, const float *bias, const void *w_bits, const int32_t *thr, void *y_bits,
+                    int B, int H, int W, int C_in, int R, int C_out, void *stream)
+{
+    if (!x || !w_bits || !thr || !y_bits) return BCNN_ERR_INVALID_ARG;
+    if (B <= 0 || H <= 0 || W <= 0 || C_in <= 0 || R <= 0 || C_out <= 0) return BCNN_ERR_INVALID_ARG;
+    if (C_in != 4 || R != 8 || C_out != 32) return BCNN_ERR_UNSUPPORTED;
+    if (!aligned16(x) || !aligned16(w_bits) || !aligned16(thr) || !aligned16(y_bits) || (bias && !aligned16(bias)))
+        return BCNN_ERR_ALIGNMENT;
+    const long npix = (long)B * H * W;
+    if (npix >= (1L << 40)) return BCNN_ERR_UNSUPPORTED;
+    return launch_stem_c4r8_k32(x, bias, static_cast<const uint32_t *>(w_bits), thr, static_cast<uint32_t *>(y_bits),
+                                npix, static_cast<cudaStream_t>(stream));
+}
+
 int bcnn_gemm_b1(const void *A_bits, const void *W_bits, int32_t *C, int64_t M, int N, int K, void *stream)
 {
     return bcnn_gemm_b1_engine(BCNN_ENGINE_AUTO, A_bits, W_bits, nullptr, C, M, N, K, stream);

@@ -62,6 +62,8 @@ __device__ __forceinline__ RowCoord row_coord(const ConvProblem &p, int m)
 
 int launch_pack(const float *x, const float *bias, uint32_t *out, long npix, int C_in, int R,
                 cudaStream_t stream);
+int launch_stem_c4r8_k32(const float *x, const float *bias, const uint32_t *w, const int32_t *thr, uint32_t *out,
+                         long npix, cudaStream_t stream);
 int launch_conv_lop3(const ConvProblem &p, cudaStream_t stream);
 bool conv_lop3_pointwise_k32(const ConvProblem &p);   // the shape runs the one-word pointwise kernel
 int launch_conv_mma_b1(const ConvProblem &p, cudaStream_t stream);

@@ -205,6 +205,69 @@ def test_pack_stem_nonfinite_and_tied_biases(bk, oracle):
         assert np.array_equal(synth.unpack_bits(out.cpu().numpy().reshape(B, H, W, 4)), want), kind
 
 
+def _stem_want(oracle, x, bias, w, thr):
+    """pack (bias, sign, 8x replication) -> binary 1x1 convolution -> threshold, all by the oracle."""
+    return oracle.threshold(oracle.conv2d(oracle.binarize(x, bias, 8), w, 1, 0), thr)
+
+
+def _run_stem(bk, x, bias, w, thr):
+    B, H, W, _ = x.shape
+    n = B * H * W * 4
+    raw, out = guard_alloc(n)
+    bk.bcnn_stem_fused(dev(x), None if bias is None else dev(bias), dev(synth.pack_bits(w)), dev(thr), out,
+                       B, H, W, 4, 8, 32)
+    torch.cuda.synchronize()
+    check_guards(raw, n)
+    return synth.unpack_bits(out.cpu().numpy().reshape(B, H, W, 4))
+
+
+@pytest.mark.parametrize("case", ["normal", "no_bias", "ties", "inf_bias", "nan_bias", "extreme_thr", "one_pixel"])
+def test_stem_fused(bk, oracle, case):
+    # fused pack + first binary 1x1 layer against the oracle's three steps; special inputs, tied and
+    # non-finite biases (the plain path), thresholds at and beyond the reachable sums
+    rng = np.random.default_rng(9100 + len(case))
+    B, H, W = (1, 1, 1) if case == "one_pixel" else (3, 37, 29)      # more pixels than one grid-stride pass of a CTA
+    x = synth.real_input(rng, (B, H, W, 4))
+    flat = x.reshape(-1)
+    if flat.size >= 12:
+        flat[:12] = [0.0, -0.0, np.inf, -np.inf, np.nan, 1e-45, -1e-45, 0.5, -0.5, 1.0, -1.0, 2.0]
+    bias = synth.real_input(rng, (32,))
+    w = synth.pm1(rng, (32, 1, 1, 32))
+    thr = synth.thresholds(rng, 32, 32)
+    if case == "no_bias":
+        bias = None
+    elif case == "ties":
+        bias[:] = np.repeat(np.array([0.5, -0.5, 0.0, -0.0], np.float32), 8)
+        if flat.size > 21:
+            bias[5] = -flat[21]                     # exact tie x + b == 0 on one channel
+        thr[:] = np.arange(-32, 32, 2, dtype=np.int32)          # every even sum is hit exactly by some output
+    elif case == "inf_bias":
+        bias[3], bias[10] = np.inf, -np.inf
+    elif case == "nan_bias":
+        bias[7] = np.nan
+    elif case == "extreme_thr":
+        thr[:8] = [-2**31, 2**31 - 1, -33, -32, 32, 33, 34, -34]
+        thr[8:16] = np.arange(-7, 9, 2)             # odd thresholds: never a tie
+    got = _run_stem(bk, x, bias, w, thr)
+    assert np.array_equal(got, _stem_want(oracle, x, bias, w, thr)), case
+    assert bk.bcnn_device_error() == 0
+
+
+def test_stem_fused_errors(bk):
+    a = torch.zeros(4096, dtype=torch.uint8, device="cuda")
+    f = torch.zeros(1024, dtype=torch.float32, device="cuda")
+    with pytest.raises(bk.BcnnError) as e:
+        bk.bcnn_stem_fused(f, None, a, a, a, 1, 4, 4, 8, 4, 32)      # not the stem shape
+    assert e.value.status == -2
+    with pytest.raises(bk.BcnnError) as e:
+        bk.bcnn_stem_fused(f, None, a[4:], a, a, 1, 4, 4, 4, 8, 32)
+    assert e.value.status == -3
+    with pytest.raises(bk.BcnnError):
+        bk.bcnn_stem_fused(f, None, a, None, a, 1, 4, 4, 4, 8, 32)
+    torch.cuda.synchronize()
+    assert int(a.sum()) == 0
+
+
 def test_pack_weights_layout(bk, oracle):
     # packing real weights [C_out][kh][kw][C_in] with the same call gives the conv weight layout
     rng = np.random.default_rng(77)

@@ -149,6 +149,27 @@ def test_backbone18_with_pack_stage_and_graph(bk, oracle):
     assert bk.bcnn_device_error() == 0
 
 
+def test_backbone18_stem_fused_full_batch(bk, oracle):
+    # the fused stem (pack + L1) at the benchmark's size, batch 256: the oracle's three steps on 300000
+    # sampled pixels plus the first and last 4096 (a 1x1 layer: every pixel is independent)
+    B = wl.BACKBONE18_BATCH
+    H, W, C, R = wl.BACKBONE18_INPUT
+    rng = synth.rng_for(5, 4321)
+    x = synth.real_input(rng, (B, H, W, C))
+    bias = synth.real_input(rng, (C * R,))
+    _, ws, ts = _chain_inputs(5, wl.BACKBONE18[:1], 1)
+    out = torch.empty(B * H * W * 4, dtype=torch.uint8, device="cuda")
+    bk.bcnn_stem_fused(dev(x), dev(bias), dev(ws[0]), dev(ts[0]), out, B, H, W, C, R, 32)
+    torch.cuda.synchronize()
+    got = out.cpu().numpy().reshape(-1, 4)
+    npix = B * H * W
+    idx = np.unique(np.concatenate([np.arange(4096), np.arange(npix - 4096, npix), rng.integers(0, npix, 300000)]))
+    xs = x.reshape(-1, C)[idx].reshape(1, -1, 1, C)
+    want = oracle.threshold(oracle.conv2d(oracle.binarize(xs, bias, R), synth.unpack_bits(ws[0]), 1, 0), ts[0])
+    assert np.array_equal(synth.unpack_bits(got[idx]), want.reshape(-1, 32))
+    assert bk.bcnn_device_error() == 0
+
+
 def test_backbone18_from_host_pipeline(bk, oracle):
     # the host-input entry of the chain: three different inputs in a row through the double-buffered
     # copy stream; every result must be the one of its own input (checked against the oracle)
