@@ -1,20 +1,20 @@
 // Weight-stationary variant of the tcgen05 engine for layers with few output channels and a
 // short K (C_out <= 128 and the expanded weights fit in shared memory).
 //
-// Same arithmetic as conv_tc_i8.cu: sign bits are expanded to bytes on chip (activations to
-// {0, 2^j}, weights to {0, 2^(7-j)}, byte 4j+i of a 32-bit group carrying bit j+8i), every
-// product of two set bits is 128, accumulators are int32 in tensor memory and
-//   sum a*g = K - 2*popc(A) - 2*popc(G) + 4*popc(A and G).
-// Differences, all aimed at short tiles (a 128 x 32 x 32 tile is one MMA instruction):
+// Arithmetic.  Sign bits are expanded to bytes on chip; byte 4j+i of a 32-bit group carries bit j+8i.
+//   activations (unsigned bytes): 0 where the bit is clear, else 2^j (j <= 6) or 64 (j = 7)
+//   weights     (signed bytes):   +-2^(6-j) (j <= 6) or +-1 (j = 7), sign = the weight's sign
+// Every product with a set activation bit is +-64, accumulators are int32 in tensor memory, and with
+// S = sum over set activation bits of the weight signs (acc = 64 S):
+//   sum a*g = 2 S + K - 2 popc(G)          (a, g in {-1,+1})
+// so the epilogue needs one constant per output channel and nothing per row.
+// Differences to conv_tc_i8.cu, all aimed at short tiles (a 128 x 32 x 32 tile is one MMA instruction):
 //   * the CTA expands its weight tile ONCE into shared memory and keeps it for all its
 //     output tiles; only activations stream through the ring;
 //   * the activation ring lives in TENSOR memory, not shared memory: producers write expanded rows
 //     with tcgen05.st and the MMA takes its A operand from tensor memory.  A narrow MMA is bound by
 //     operand fetch from shared memory (128 x 32 bytes of A per instruction whatever N is); with A in
 //     tensor memory only the small weight slice is fetched;
-//   * one extra all-ones weight row is appended, so column BN of every accumulator holds
-//     128 * popc(A) for its row: the epilogue reads the row popcount from tensor memory and
-//     no per-tile constants travel through shared memory;
 //   * G producer groups of 128 threads take the ring's stages round-robin, so that G stages
 //     are being gathered / expanded at any time (one thread's stage latency is several
 //     hundred cycles, an MMA stage as little as 64);
@@ -43,7 +43,7 @@ constexpr int ERR_EPILOGUE_TIMEOUT = 113;
 
 // DUAL: two CTAs share an SM (two independent MMA issuers), each with half of tensor memory.
 template <int BN, int G, bool DUAL> struct Cfg {
-    static constexpr int BNX = BN + 16;                       // + the all-ones row (MMA N is a multiple of 16)
+    static constexpr int BNX = BN;
     static constexpr int PROD_THREADS = G * BM;
     // Tensor memory (512 columns): NBUF accumulator buffers of BNX columns, then the activation ring,
     // one stage = 128 rows x 128 expanded bytes = 32 columns.
@@ -143,30 +143,29 @@ conv_tc_ws_kernel(const ConvProblem p)
     }
 
     // ---- one-off: expand the weight tile (+ the all-ones row), column constants, K-word table
-    for (int idx = tid; idx < ktiles * BNX; idx += C::THREADS) {
-        const int kt = idx / BNX, row = idx - kt * BNX;
-        uint32_t w[4];
+    for (int idx = tid; idx < ktiles * BN; idx += C::THREADS) {
+        const int kt = idx / BN, row = idx - kt * BN;
+        const uint32_t row_addr = wexp + (uint32_t)kt * C::W_TILE_BYTES + (uint32_t)row * ROWB;
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
             const int kword = kt * 4 + e;
-            uint32_t v = 0;
-            if (kword < p.kwords) {
-                if (row < BN) v = (row < p.C_out) ? __ldg(p.w + (long)row * p.kwords + kword) : 0u;
-                else if (row == BN) v = 0xffffffffu;
-            }
-            w[e] = v;
+            const bool live = kword < p.kwords && row < p.C_out;         // rows / K words beyond the problem: zero bytes
+            const uint32_t w = live ? __ldg(p.w + (long)row * p.kwords + kword) : 0u;
+            expand_store_w_signed(w, live, row_addr, row & 7, 2 * e);
         }
-        const uint32_t row_addr = wexp + (uint32_t)kt * C::W_TILE_BYTES + (uint32_t)row * ROWB;
-#pragma unroll
-        for (int e = 0; e < 4; ++e) expand_store_w(w[e], row_addr, row & 7, 2 * e);
     }
     for (int c = tid; c < BN; c += C::THREADS) {
         int pop = 0;
         if (c < p.C_out)
             for (int kw = 0; kw < p.kwords; ++kw) pop += __popc(__ldg(p.w + (long)c * p.kwords + kw));
-        // with acc = 128*popc(A and G), pa = popc(A):  int32: (acc >> 5) - 2*pa + (K - 2*pop)
-        //                                             fused: acc - 64*pa - 32*(thr - K + 2*pop) >= 0
-        const int cst = FUSED ? -32 * ((c < p.C_out ? __ldg(p.thr + c) : 0) - p.K + 2 * pop) : p.K - 2 * pop;
+        // with acc = 64 * S:   int32: (acc >> 5) + (K - 2*pop)      fused: acc + 32*(K - 2*pop - thr) >= 0
+        // (a threshold beyond +-(K + 1) decides like that bound; clamping keeps the constant inside int32)
+        int cst = p.K - 2 * pop;
+        if (FUSED) {
+            int t = c < p.C_out ? __ldg(p.thr + c) : 0;
+            t = max(min(t, p.K + 1), -p.K - 1);
+            cst = 32 * (cst - t);
+        }
         asm volatile("st.shared.b32 [%0], %1;" ::"r"(colc_addr + 4u * c), "r"(cst) : "memory");
     }
     const int gw = gather_width(p.cw);
@@ -185,7 +184,7 @@ conv_tc_ws_kernel(const ConvProblem p)
         // stage at a time through named barrier 1 + slot.  There is one issuer on purpose: the
         // producers' parity waits rely on the ring being consumed in order (a second issuer working on
         // the next tile lets a late slot fall two phases behind a waiting producer).
-        constexpr uint32_t idesc = make_idesc(BNX);
+        constexpr uint32_t idesc = make_idesc(BNX) | (1u << 10);                  // B operand: signed bytes
         const uint64_t desc0 = make_desc(0);
         const uint32_t desc_hi = (uint32_t)(desc0 >> 32);
         const uint32_t tmem_u = __shfl_sync(0xffffffffu, tmem_base, 0);             // warp-uniform copy for the issuer
@@ -251,7 +250,6 @@ conv_tc_ws_kernel(const ConvProblem p)
             if (!alive) break;
             tc_fence_after();
             const uint32_t t_addr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(buf * BNX);
-            const uint32_t pa128 = tc_ld1(t_addr + BN);        // 128 * popc(A) of this row
             uint32_t words[BN / 32];
 #pragma unroll
             for (int ch = 0; ch < BN / 32; ++ch) {
@@ -261,29 +259,27 @@ conv_tc_ws_kernel(const ConvProblem p)
                     uint32_t v[32];
                     tc_ld32(t_addr + (uint32_t)col0, v);
                     if (FUSED) {
-                        const int rowc = -(int)(pa128 >> 1);          // -64 * popc(A)
                         uint32_t acc = 0;
 #pragma unroll
                         for (int i4 = 7; i4 >= 0; --i4) {
                             const uint4 cc = ld_shared_v4(colc_addr + 4u * (col0 + 4 * i4));
-                            acc = __funnelshift_l((uint32_t)((int)v[4 * i4 + 3] + rowc + (int)cc.w), acc, 1);
-                            acc = __funnelshift_l((uint32_t)((int)v[4 * i4 + 2] + rowc + (int)cc.z), acc, 1);
-                            acc = __funnelshift_l((uint32_t)((int)v[4 * i4 + 1] + rowc + (int)cc.y), acc, 1);
-                            acc = __funnelshift_l((uint32_t)((int)v[4 * i4 + 0] + rowc + (int)cc.x), acc, 1);
+                            acc = __funnelshift_l((uint32_t)((int)v[4 * i4 + 3] + (int)cc.w), acc, 1);
+                            acc = __funnelshift_l((uint32_t)((int)v[4 * i4 + 2] + (int)cc.z), acc, 1);
+                            acc = __funnelshift_l((uint32_t)((int)v[4 * i4 + 1] + (int)cc.y), acc, 1);
+                            acc = __funnelshift_l((uint32_t)((int)v[4 * i4 + 0] + (int)cc.x), acc, 1);
                         }
                         words[ch] = ~acc;
                     } else if (em < p.M) {
-                        const int rowc = -(int)(pa128 >> 6);          // -2 * popc(A)
                         int32_t *dst = static_cast<int32_t *>(p.out) + (long)em * p.C_out + col0;
                         const bool vec = (p.C_out & 3) == 0 && (col0 + 32 <= p.C_out);
 #pragma unroll
                         for (int i4 = 0; i4 < 8; ++i4) {
                             const uint4 cc = ld_shared_v4(colc_addr + 4u * (col0 + 4 * i4));
                             int4 o;
-                            o.x = (int)(v[4 * i4 + 0] >> 5) + rowc + (int)cc.x;
-                            o.y = (int)(v[4 * i4 + 1] >> 5) + rowc + (int)cc.y;
-                            o.z = (int)(v[4 * i4 + 2] >> 5) + rowc + (int)cc.z;
-                            o.w = (int)(v[4 * i4 + 3] >> 5) + rowc + (int)cc.w;
+                            o.x = ((int)v[4 * i4 + 0] >> 5) + (int)cc.x;
+                            o.y = ((int)v[4 * i4 + 1] >> 5) + (int)cc.y;
+                            o.z = ((int)v[4 * i4 + 2] >> 5) + (int)cc.z;
+                            o.w = ((int)v[4 * i4 + 3] >> 5) + (int)cc.w;
                             if (vec) {
                                 *reinterpret_cast<int4 *>(dst + 4 * i4) = o;
                             } else {
@@ -372,13 +368,11 @@ conv_tc_ws_kernel(const ConvProblem p)
                 if (c_src == bits_end) c_src = bits0;
                 if (!mbar_wait_warp(empty_bar(s), phase, abort_flag, p.err, ERR_PRODUCER_TIMEOUT)) break;
                 tc_fence_after();     // the MMAs that read this slot are complete (their commit released it)
-                // expanded row -> 32 columns of this lane: column 8*e + j = word j of K word e (bytes 0 or 2^j)
+                // expanded row -> 32 columns of this lane: column 8*e + j = word j of K word e (bytes 0 or 2^j, 64 for j = 7)
                 uint32_t v[32];
                 const uint32_t wds[4] = {bits.x, bits.y, bits.z, bits.w};
 #pragma unroll
-                for (int e = 0; e < 4; ++e)
-#pragma unroll
-                    for (int j = 0; j < 8; ++j) v[8 * e + j] = wds[e] & (0x01010101u << j);
+                for (int e = 0; e < 4; ++e) expand_a(wds[e], &v[8 * e]);
                 tc_st32(st_addr0 + (uint32_t)s * 32u, v);
                 tc_fence_before();
                 __syncwarp();
@@ -437,9 +431,7 @@ conv_tc_ws_kernel(const ConvProblem p)
                         uint32_t v[32];
                         const uint32_t wds[4] = {bits.x, bits.y, bits.z, bits.w};
 #pragma unroll
-                        for (int e = 0; e < 4; ++e)
-#pragma unroll
-                            for (int j = 0; j < 8; ++j) v[8 * e + j] = wds[e] & (0x01010101u << j);
+                        for (int e = 0; e < 4; ++e) expand_a(wds[e], &v[8 * e]);
                         tc_st32(st_addr0 + (uint32_t)s * 32u, v);
                         tc_fence_before();
                         __syncwarp();

@@ -146,6 +146,28 @@ __device__ __forceinline__ void tc_st32(uint32_t taddr, const uint32_t (&v)[32])
           "r"(v[24]), "r"(v[25]), "r"(v[26]), "r"(v[27]), "r"(v[28]), "r"(v[29]), "r"(v[30]), "r"(v[31])
         : "memory");
 }
+// Same without the completion wait, for several stores followed by one tc_wait_st().
+__device__ __forceinline__ void tc_st32_nowait(uint32_t taddr, const uint32_t (&v)[32])
+{
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+        "{%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,"
+        "%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32};"
+        ::"r"(taddr),
+          "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7]),
+          "r"(v[8]), "r"(v[9]), "r"(v[10]), "r"(v[11]), "r"(v[12]), "r"(v[13]), "r"(v[14]), "r"(v[15]),
+          "r"(v[16]), "r"(v[17]), "r"(v[18]), "r"(v[19]), "r"(v[20]), "r"(v[21]), "r"(v[22]), "r"(v[23]),
+          "r"(v[24]), "r"(v[25]), "r"(v[26]), "r"(v[27]), "r"(v[28]), "r"(v[29]), "r"(v[30]), "r"(v[31])
+        : "memory");
+}
+// 8 columns (one K word) of this warp's 32 lanes <- 8 registers.
+__device__ __forceinline__ void tc_st8_nowait(uint32_t taddr, const uint32_t (&v)[8])
+{
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};"
+                 ::"r"(taddr), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]), "r"(v[5]), "r"(v[6]), "r"(v[7])
+                 : "memory");
+}
+__device__ __forceinline__ void tc_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tc_commit_pred(uint32_t bar, uint32_t pred)
 {
     asm volatile(
@@ -229,6 +251,32 @@ __device__ __forceinline__ void expand_store_w(uint32_t w, uint32_t row_addr, in
                  r & 0x80808080u, r & 0x40404040u, r & 0x20202020u, r & 0x10101010u);
     st_shared_v4(row_addr + (uint32_t)(((c + 1) ^ xr) << 4),
                  r & 0x08080808u, r & 0x04040404u, r & 0x02020202u, r & 0x01010101u);
+}
+
+// Activation word -> 8 words for the signed-weight scheme: word j holds bits j, j+8, j+16, j+24 as bytes
+// 2^j for j <= 6; bit 7 goes to 64 as well (its weight magnitude is 1 where bit 6's is 1 too, see below).
+__device__ __forceinline__ void expand_a(uint32_t w, uint32_t *v)
+{
+#pragma unroll
+    for (int j = 0; j < 7; ++j) v[j] = w & (0x01010101u << j);
+    v[7] = (w >> 1) & 0x40404040u;
+}
+// Weight word -> signed bytes matching expand_a: magnitude 2^(6-j) for j <= 6 and 1 for j = 7, sign = the weight's
+// sign (bit set: +), so that every product with a set activation byte is +-64.  `live` false writes zeros.
+// The bits of each byte are reversed once (bit j -> bit 7-j) and inverted; in word j the flag "weight is -" then
+// sits at bit 7-j of every byte, exactly the lowest bit of the two's-complement pattern of -2^(6-j) above the
+// magnitude bit: flag * (2^(j+1) - 1) sets bits 7-j..7, adding the magnitude bit 6-j completes the byte (no
+// carries between bytes: every byte stays below 256).  Word 7 (magnitude 1): flag at bit 0, * 0xFE, + 1.
+__device__ __forceinline__ void expand_store_w_signed(uint32_t w, bool live, uint32_t row_addr, int xr, int c)
+{
+    const uint32_t nr = ~__byte_perm(__brev(w), 0u, 0x0123u);
+    uint32_t o[8];
+#pragma unroll
+    for (int j = 0; j < 7; ++j)
+        o[j] = live ? (nr & (0x01010101u << (7 - j))) * ((2u << j) - 1u) + (0x01010101u << (6 - j)) : 0u;
+    o[7] = live ? (nr & 0x01010101u) * 0xFEu + 0x01010101u : 0u;
+    st_shared_v4(row_addr + (uint32_t)(((c) ^ xr) << 4), o[0], o[1], o[2], o[3]);
+    st_shared_v4(row_addr + (uint32_t)(((c + 1) ^ xr) << 4), o[4], o[5], o[6], o[7]);
 }
 
 // ---- implicit-im2col gather -----------------------------------------------------------------------
