@@ -471,9 +471,88 @@ def run_sweep(args):
     return 0 if err == 0 else 1
 
 
+def run_paper1x1(args):
+    """The paper's own binary workload (not the headline line): the 32 binary 1x1 convolutions of the
+    network of Table 1 (2.41e9 binary MACs per image; 64 convolutions for P = 2 parallel branches), each
+    with the fused threshold epilogue, on independent seeded inputs (the real-valued depth-wise / batch
+    norm / PReLU steps between them are outside the binary hot path).  One step = all convolutions for
+    one batch, replayed from a CUDA graph.  Prints one JSON line."""
+    import torch
+    from paper_2010_00704_b200 import build, binding
+    build.build()
+    binding.load()
+    torch.cuda.set_device(0)
+    B, P = args.batch, args.branches
+    convs = wl.paper_binary_1x1_convs(P)
+    jobs = []
+    for li, (l, count) in enumerate(convs):
+        rng = synth.rng_for(6, li)
+        x = torch.from_numpy(synth.random_bits(rng, (l.in_bytes(B),))).cuda()
+        for c in range(count):
+            Wb = torch.from_numpy(synth.random_bits(rng, (l.w_bytes(),))).cuda()
+            thr = torch.from_numpy(synth.thresholds(rng, l.K, l.C_out)).cuda()
+            out = torch.empty(l.out_bits_bytes(B), dtype=torch.uint8, device="cuda")
+            jobs.append((l, x, Wb, thr, out))
+
+    def launch(j):
+        l, x, Wb, thr, out = j
+        binding.bcnn_conv2d_b1_fused(x, Wb, thr, out, B, l.H, l.W, l.C_in, l.C_out, 1, 1, 1, 0)
+
+    def step():
+        for j in jobs:
+            launch(j)
+
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        step()
+    torch.cuda.current_stream().wait_stream(side)
+    torch.cuda.synchronize()
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        step()
+    for _ in range(max(args.warmup, 3)):
+        g.replay()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(args.steps):
+        g.replay()
+    e1.record()
+    torch.cuda.synchronize()
+    ms_step = e0.elapsed_time(e1) / args.steps
+    # per shape: CUDA events around each launch, averaged
+    per = {}
+    for _ in range(args.steps):
+        for j in jobs:
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            launch(j)
+            b.record()
+            per.setdefault(j[0].name, []).append((a, b))
+    torch.cuda.synchronize()
+    shapes = []
+    for l, count in convs:
+        ms = float(np.mean([a.elapsed_time(b) for a, b in per[l.name]]))
+        shapes.append({"layer": l.name, "count": count, "M": l.M(B), "N": l.C_out, "K": l.K,
+                       "engine": binding.bcnn_auto_engine(B, l.H, l.W, l.C_in, l.C_out, 1, 1, 1, 0),
+                       "ms_per_launch": ms, "tops": l.ops(B) / (ms / 1e3) / 1e12,
+                       "gbs": (l.in_bytes(B) + l.out_bits_bytes(B)) / (ms / 1e3) / 1e9})
+    err = binding.bcnn_device_error()
+    ops = 2 * sum(n * l.macs(B) for l, n in convs)
+    print(json.dumps({
+        "mode": "paper1x1", "metric": "binary conv throughput (2*M*N*K bit-ops/s), the paper's 1x1 convolutions (Table 1)",
+        "value": ops / (ms_step / 1e3) / 1e12, "unit": UNIT, "ms_per_step": ms_step, "images_per_s": B / (ms_step / 1e3),
+        "binary_macs_per_image": ops // (2 * B), "n_gpus": 1, "steps": args.steps, "data": "synthetic",
+        "config": {"workload": f"Table 1 network, binary 1x1 convolutions only, P = {P}, batch {B}", "launches": len(jobs),
+                   "launch": "CUDA graph replay"},
+        "per_shape": shapes, "device_error": err}))
+    return 0 if err == 0 else 1
+
+
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("--mode", default="bench", choices=["bench", "sweep"])
+    ap.add_argument("--mode", default="bench", choices=["bench", "sweep", "paper1x1"])
     ap.add_argument("--engines", default="auto,lop3,mma_b1,tc_i8,mma_s8,tc_ws")
     ap.add_argument("--sweep-set", default="all", choices=["gemm", "conv", "all"])
     ap.add_argument("--only", default="", help="sweep mode: run only shapes whose label contains this text")
@@ -483,11 +562,15 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--batch", type=int, default=256, help="paper1x1 mode: images per step")
+    ap.add_argument("--branches", type=int, default=1, choices=[1, 2], help="paper1x1 mode: parallel binary branches P")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)
     if args.mode == "sweep":
         return run_sweep(args)
+    if args.mode == "paper1x1":
+        return run_paper1x1(args)
     return run_gpu(args)
 
 

@@ -168,3 +168,25 @@ def paper_table1_binary_counts(P: int = 1):
                 params += C * C
                 macs += hw_out * C * C
     return P * params, P * macs
+
+
+def paper_binary_1x1_convs(P: int = 1):
+    """The binary 1x1 convolutions of the network of Table 1 as (ConvLayer, count) pairs, in network order.
+
+    Same rules as ``paper_table1_binary_counts``: per block one C x C conv at the block's input resolution
+    (S * res) and one at its output resolution, plus one more at the output resolution on the identity
+    path of a replicate / down-sampling block; P parallel branches repeat every conv P times
+    (Section 4.2.1).  Their MACs add up to the paper's 2.41e9 (4.83e9 for P = 2) per image.
+    """
+    out = []
+    for name, blocks, S, R, C, res in PAPER_TABLE1:
+        if blocks == 0:
+            continue
+        special = (R > 1) or (S > 1)
+        tag = name.replace(" ", "_")
+        if S > 1:
+            out.append((ConvLayer(f"{tag}_in{res * S}_c{C}", res * S, res * S, C, C, 1, 1, 0), P * blocks))
+            out.append((ConvLayer(f"{tag}_out{res}_c{C}", res, res, C, C, 1, 1, 0), P * blocks * (2 if special else 1)))
+        else:
+            out.append((ConvLayer(f"{tag}_{res}_c{C}", res, res, C, C, 1, 1, 0), P * blocks * (3 if special else 2)))
+    return out

@@ -195,3 +195,32 @@ def test_backbone18_from_host_pipeline(bk, oracle):
         got = synth.unpack_bits(oh.numpy().reshape(B, 7, 7, 512 // 8))
         assert np.array_equal(got[:1], cur)
     assert bk.bcnn_device_error() == 0
+
+
+@pytest.mark.parametrize("li", range(14))
+def test_paper_1x1_convs(bk, oracle, li):
+    # every distinct binary 1x1 convolution of the paper's own network (Table 1) at batch 4, fused and int32:
+    # the definition oracle on 512 sampled pixels plus the first and last 128, the packed checker on every output
+    l, _count = wl.paper_binary_1x1_convs(1)[li]
+    B = 4
+    rng = synth.rng_for(6, li)
+    xb = synth.random_bits(rng, (B, l.H, l.W, l.C_in // 8))
+    wb = synth.random_bits(rng, (l.C_out, 1, 1, l.C_in // 8))
+    thr = synth.thresholds(rng, l.K, l.C_out)
+    M, N = l.M(B), l.C_out
+    y = torch.empty(M * N, dtype=torch.int32, device="cuda")
+    yb = torch.empty(M * N // 8, dtype=torch.uint8, device="cuda")
+    bk.bcnn_conv2d_b1(dev(xb), dev(wb), y, B, l.H, l.W, l.C_in, N, 1, 1, 1, 0)
+    bk.bcnn_conv2d_b1_fused(dev(xb), dev(wb), dev(thr), yb, B, l.H, l.W, l.C_in, N, 1, 1, 1, 0)
+    torch.cuda.synchronize()
+    got = y.cpu().numpy().reshape(M, N)
+    got_bits = yb.cpu().numpy().reshape(M, N // 8)
+    full = oracle.checker_conv2d(xb, wb, (B, l.H, l.W, l.C_in, N, 1, 1), 1, 0).reshape(M, N)
+    assert np.array_equal(got, full)
+    assert np.array_equal(got_bits, synth.pack_bits(np.where(full >= thr[None, :], 1, -1).astype(np.int8)))
+    rows = np.unique(np.concatenate([np.arange(min(128, M)), np.arange(max(0, M - 128), M), rng.integers(0, M, 512)]))
+    xs = synth.unpack_bits(xb.reshape(M, l.C_in // 8)[rows]).reshape(1, -1, 1, l.C_in)
+    want = oracle.conv2d(xs, synth.unpack_bits(wb), 1, 0).reshape(-1, N)
+    assert np.array_equal(got[rows], want)
+    assert np.array_equal(synth.unpack_bits(got_bits[rows]), oracle.threshold(want, thr))
+    assert bk.bcnn_device_error() == 0

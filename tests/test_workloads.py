@@ -45,3 +45,17 @@ def test_workload_shapes():
         assert (prev.OH, prev.OW, prev.C_out) == (nxt.H, nxt.W, nxt.C_in)
     assert wl.BACKBONE18[2] == wl.STEM_DOWN[0].__class__(wl.BACKBONE18[2].name, 112, 112, 32, 64, 3, 2, 1)
     assert wl.BACKBONE18[-1].OH == 7 and wl.BACKBONE18[-1].C_out == 512
+
+
+def test_paper_1x1_conv_list_reproduces_table2():
+    # the per-layer list used as a workload must add up to the totals the paper prints
+    for P in (1, 2):
+        convs = wl.paper_binary_1x1_convs(P)
+        params = sum(n * l.C_in * l.C_out for l, n in convs)
+        macs = sum(n * l.macs(1) for l, n in convs)
+        assert (params, macs) == wl.paper_table1_binary_counts(P)
+    convs = wl.paper_binary_1x1_convs(1)
+    assert sum(n for _, n in convs) == 32
+    assert all(l.k == 1 and l.C_in == l.C_out for l, _ in convs)
+    assert {l.C_in for l, _ in convs} == {32, 64, 128, 256, 512, 1024}
+    assert {l.H for l, _ in convs} == {224, 112, 56, 28, 14, 7}
