@@ -12,7 +12,10 @@ Parity pins (see tests/test_oracle_pins.py): closed forms for constant inputs
 including the border values that depend on the -1 padding, a one-hot weight case
 worked by hand, brute force in pure Python on tiny shapes, the textbook library
 convolution of the padded +-1 tensors, the xor/popcount identity against a float
-dot product, and the tie rule of the threshold.  The paper prints no worked
+dot product, and the tie rule of the threshold; for the convolution module (batch
+norm, identity, PReLU, fp16 store, next sign) a case worked by hand, the fp16
+round-to-even ties, the sign-of-the-stored-value rule, the reduction to the integer
+threshold and the elementwise numpy restatement.  The paper prints no worked
 numeric example of a convolution, so beyond those pins parity is unpinned by the
 paper itself.
 """
@@ -157,6 +160,32 @@ def threshold(acc: np.ndarray, thr: np.ndarray) -> np.ndarray:
     rows = acc.size // N if N else 0
     _load().oracle_threshold(_ptr(acc), _ptr(thr), _ptr(out), ctypes.c_long(rows), ctypes.c_long(N))
     return out
+
+
+def conv_module(acc: np.ndarray, scale, shift, identity, slope, next_bias=None, want_sign: bool = True):
+    """Batch norm (scale, shift) -> + identity (fp16) -> PReLU -> fp16 real map, and the next module's
+    sign(stored value + next_bias) as int8 +-1 (Section 4.2.1).  acc int32 [..., N]; per-channel fp32
+    vectors of length N; identity float16 [..., N] or None.  Returns (y float16, s int8 or None)."""
+    acc = _c(acc, np.int32)
+    N = acc.shape[-1]
+    scale, shift, slope = _c(scale, np.float32), _c(shift, np.float32), _c(slope, np.float32)
+    assert scale.shape == (N,) and shift.shape == (N,) and slope.shape == (N,)
+    iptr = None
+    if identity is not None:
+        identity = _c(identity, np.float16)
+        assert identity.shape == acc.shape
+        iptr = _ptr(identity)
+    nptr = None
+    if next_bias is not None:
+        next_bias = _c(next_bias, np.float32)
+        assert next_bias.shape == (N,)
+        nptr = _ptr(next_bias)
+    y = np.empty(acc.shape, dtype=np.float16)
+    s = np.empty(acc.shape, dtype=np.int8) if want_sign else None
+    rows = acc.size // N if N else 0
+    _load().oracle_conv_module(_ptr(acc), _ptr(scale), _ptr(shift), iptr, _ptr(slope), nptr, _ptr(y),
+                               None if s is None else _ptr(s), ctypes.c_long(rows), ctypes.c_long(N))
+    return y, s
 
 
 # ---- bit-packed checker (not the oracle; proven equal to it by the CPU tests) ----

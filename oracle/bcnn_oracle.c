@@ -33,6 +33,7 @@
  */
 #include <stdint.h>
 #include <stddef.h>
+#include <string.h>
 
 #ifdef _OPENMP
 #include <omp.h>
@@ -181,4 +182,42 @@ void oracle_threshold(const int32_t *acc, const int32_t *thr, int8_t *out,
     for (long i = 0; i < rows; ++i)
         for (long n = 0; n < N; ++n)
             out[i * N + n] = (acc[i * N + n] >= thr[n]) ? (int8_t)1 : (int8_t)-1;
+}
+
+/*
+ * The convolution module around a binary convolution (Section 4.2.1, Figure 4 top), applied to the
+ * convolution's integer result acc:
+ *   t = acc * scale[n] + shift[n]          batch norm as a per-channel scale and bias
+ *   u = t + identity                       the module's real input, carried around the binary conv
+ *   r = (u >= 0) ? u : slope[n] * u        PReLU with a per-channel slope
+ *   y = fp16(r)                            the real feature map as it is stored
+ *   s = (y + next_bias[n] >= 0) ? +1 : -1  the next module's bias + sign, taken of the STORED value
+ * Every step is one fp32 operation rounded to nearest even (no fused multiply-add: this file is
+ * compiled with -ffp-contract=off); the conversion to fp16 rounds to nearest even.  identity (fp16
+ * bit patterns, may be NULL = no identity path) and y are [rows][N]; s may be NULL.
+ */
+void oracle_conv_module(const int32_t *acc, const float *scale, const float *shift,
+                        const uint16_t *identity, const float *slope, const float *next_bias,
+                        uint16_t *y, int8_t *s, long rows, long N)
+{
+#pragma omp parallel for schedule(static)
+    for (long i = 0; i < rows; ++i)
+        for (long n = 0; n < N; ++n) {
+            const long k = i * N + n;
+            float t = (float)acc[k] * scale[n];
+            t = t + shift[n];
+            float u = t;
+            if (identity) {
+                _Float16 hi;
+                memcpy(&hi, &identity[k], sizeof hi);
+                u = t + (float)hi;
+            }
+            const float r = (u >= 0.0f) ? u : slope[n] * u;
+            const _Float16 h = (_Float16)r;
+            memcpy(&y[k], &h, sizeof h);
+            if (s) {
+                const float v = (float)h + (next_bias ? next_bias[n] : 0.0f);
+                s[k] = (v >= 0.0f) ? (int8_t)1 : (int8_t)-1;
+            }
+        }
 }

@@ -282,3 +282,84 @@ def test_pack_unpack_layout():
     assert b.tolist() == [[0x01, 0x02, 0x00, 0x00, 0x80]]
     assert b[:, :4].copy().view("<u4").tolist() == [[0x00000201]]
     assert np.array_equal(synth.unpack_bits(b), v)
+
+
+# ---- convolution module: batch norm -> + identity -> PReLU -> fp16 store -> next sign (Section 4.2.1) ----
+
+def test_conv_module_hand_worked(oracle):
+    # four channels worked by hand with exactly representable numbers:
+    #   c0: 3*0.5 + 0.25 = 1.75, + 1 = 2.75 (>= 0 stays);           sign(2.75 - 3) = -1
+    #   c1: -3*0.5 + 0.25 = -1.25, + 1 = -0.25, * 0.25 = -0.0625;   sign(-0.0625 + 0.0625 = 0) = +1 (tie goes up)
+    #   c2: 0*2 - 1 = -1, + 0.5 = -0.5, * 0.125 = -0.0625;          sign(-0.0625 + 0.0625) = +1
+    #   c3: 5*(-1) + 1 = -4, - 10 = -14, * 0.5 = -7;                sign(-7 + 7) = +1
+    acc = np.array([[3, -3, 0, 5]], np.int32)
+    y, s = oracle.conv_module(acc, [0.5, 0.5, 2, -1], [0.25, 0.25, -1, 1], np.array([[1, 1, 0.5, -10]], np.float16),
+                              [0.25, 0.25, 0.125, 0.5], [-3, 0.0625, 0.0625, 7])
+    assert y.dtype == np.float16 and y.tolist() == [[2.75, -0.0625, -0.0625, -7.0]]
+    assert s.tolist() == [[-1, 1, 1, 1]]
+
+
+def test_conv_module_pass_through_and_relu(oracle):
+    # scale 1, shift 0, no identity, slope 1: the stored map is the integer sum itself (exact in fp16 up to 2048);
+    # slope 0 makes the PReLU a ReLU
+    acc = np.arange(-2048, 2049, dtype=np.int32).reshape(-1, 1)
+    one, zero = np.ones(1, np.float32), np.zeros(1, np.float32)
+    y, _ = oracle.conv_module(acc, one, zero, None, one, None, want_sign=False)
+    assert np.array_equal(y.astype(np.int32), acc)
+    y, _ = oracle.conv_module(acc, one, zero, None, zero, None, want_sign=False)
+    assert np.array_equal(y.astype(np.int32), np.maximum(acc, 0))
+
+
+def test_conv_module_fp16_ties_and_sign_of_stored_value(oracle):
+    # 2049 and 2051 lie halfway between fp16 neighbours: round to even gives 2048 and 2052;
+    # the next sign looks at the STORED value: 2049 -> 2048, and 2048 - 2048.5 < 0 although 2049 - 2048.5 > 0
+    acc = np.array([[2049], [2051], [2050]], np.int32)
+    one, zero = np.ones(1, np.float32), np.zeros(1, np.float32)
+    y, s = oracle.conv_module(acc, one, zero, None, one, np.array([-2048.5], np.float32))
+    assert y.astype(np.float32).ravel().tolist() == [2048.0, 2052.0, 2050.0]
+    assert s.ravel().tolist() == [-1, 1, 1]
+    # overflow of the fp16 range stores infinity, a NaN scale stores NaN whose sign is -1
+    y, s = oracle.conv_module(np.array([[70000]], np.int32), one, zero, None, one, zero)
+    assert np.isinf(y[0, 0]) and s[0, 0] == 1
+    y, s = oracle.conv_module(np.array([[1]], np.int32), np.array([np.nan], np.float32), zero, None, one, zero)
+    assert np.isnan(y[0, 0]) and s[0, 0] == -1
+    # negative zero (0 * -1 = -0, -0 + -0 = -0) is >= 0: it passes the PReLU unchanged and its sign is +1
+    y, s = oracle.conv_module(np.array([[0]], np.int32), np.array([-1.0], np.float32), np.array([-0.0], np.float32), None,
+                              np.array([7.0], np.float32), zero)
+    assert np.signbit(y[0, 0]) and y[0, 0] == 0 and s[0, 0] == 1
+
+
+def test_conv_module_reduces_to_the_integer_threshold(oracle):
+    # unit scale, integer shift and next bias, no identity, slope 1: sign(acc + b + nb >= 0) is the integer
+    # threshold acc >= -(b + nb) of the fused path (sums stay below 2048, exact in fp16)
+    rng = np.random.default_rng(31)
+    N = 24
+    acc = rng.integers(-900, 901, size=(50, N)).astype(np.int32)
+    b = rng.integers(-100, 101, size=N).astype(np.float32)
+    nb = rng.integers(-100, 101, size=N).astype(np.float32)
+    _, s = oracle.conv_module(acc, np.ones(N, np.float32), b, None, np.ones(N, np.float32), nb)
+    assert np.array_equal(s, oracle.threshold(acc, (-(b + nb)).astype(np.int32)))
+
+
+def test_conv_module_against_elementwise_numpy(oracle):
+    # numpy restatement, one IEEE fp32 operation per step (numpy never fuses), fp16 conversion by astype;
+    # the sign is the already pinned binarize() of the stored map
+    rng = np.random.default_rng(32)
+    N = 40
+    acc = rng.integers(-1152, 1153, size=(3, 5, 7, N)).astype(np.int32)
+    scale = rng.standard_normal(N).astype(np.float32) * np.float32(0.05)
+    shift = rng.standard_normal(N).astype(np.float32)
+    slope = rng.uniform(-0.5, 1.5, N).astype(np.float32)
+    ident = rng.standard_normal(acc.shape).astype(np.float16)
+    nb = rng.standard_normal(N).astype(np.float32)
+    y, s = oracle.conv_module(acc, scale, shift, ident, slope, nb)
+    t = acc.astype(np.float32) * scale
+    t = t + shift
+    u = t + ident.astype(np.float32)
+    r = np.where(u >= 0, u, slope * u).astype(np.float32)
+    want = r.astype(np.float16)
+    assert np.array_equal(y.view(np.uint16), want.view(np.uint16))
+    assert np.array_equal(s, oracle.binarize(want.astype(np.float32), nb, 1))
+    # planting a mistake must show: sign of the unrounded value differs somewhere on a finer grid
+    y2, _ = oracle.conv_module(acc, scale, shift, None, slope, None, want_sign=False)
+    assert not np.array_equal(y2.view(np.uint16), y.view(np.uint16))
