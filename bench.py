@@ -483,20 +483,38 @@ def run_paper1x1(args):
     binding.load()
     torch.cuda.set_device(0)
     B, P = args.batch, args.branches
+    module = args.epilogue == "module"
+    peaks = load_peaks()
     convs = wl.paper_binary_1x1_convs(P)
     jobs = []
     for li, (l, count) in enumerate(convs):
         rng = synth.rng_for(6, li)
         x = torch.from_numpy(synth.random_bits(rng, (l.in_bytes(B),))).cuda()
+        ident = yreal = None
+        if module:
+            # the module's real input (fp16 NHWC, standard normal) and its real output, shared by the repeats
+            ident = torch.randn(l.M(B) * l.C_out, dtype=torch.float16, device="cuda",
+                                generator=torch.Generator(device="cuda").manual_seed(synth.seed_for(6, li)))
+            yreal = torch.empty(l.M(B) * l.C_out, dtype=torch.float16, device="cuda")
         for c in range(count):
             Wb = torch.from_numpy(synth.random_bits(rng, (l.w_bytes(),))).cuda()
             thr = torch.from_numpy(synth.thresholds(rng, l.K, l.C_out)).cuda()
             out = torch.empty(l.out_bits_bytes(B), dtype=torch.uint8, device="cuda")
-            jobs.append((l, x, Wb, thr, out))
+            extra = None
+            if module:
+                sc = torch.from_numpy((rng.standard_normal(l.C_out) / np.sqrt(l.K)).astype(np.float32)).cuda()
+                sh, nb = (torch.from_numpy(synth.real_input(rng, (l.C_out,))).cuda() for _ in range(2))
+                sl = torch.from_numpy(rng.uniform(0.0, 0.5, l.C_out).astype(np.float32)).cuda()
+                extra = (sc, sh, ident, sl, nb, yreal)
+            jobs.append((l, x, Wb, thr, out, extra))
 
     def launch(j):
-        l, x, Wb, thr, out = j
-        binding.bcnn_conv2d_b1_fused(x, Wb, thr, out, B, l.H, l.W, l.C_in, l.C_out, 1, 1, 1, 0)
+        l, x, Wb, thr, out, extra = j
+        if module:
+            sc, sh, idn, sl, nb, yr = extra
+            binding.bcnn_conv2d_b1_module(x, Wb, sc, sh, idn, sl, nb, yr, out, B, l.H, l.W, l.C_in, l.C_out, 1, 1, 1, 0)
+        else:
+            binding.bcnn_conv2d_b1_fused(x, Wb, thr, out, B, l.H, l.W, l.C_in, l.C_out, 1, 1, 1, 0)
 
     def step():
         for j in jobs:
@@ -535,16 +553,21 @@ def run_paper1x1(args):
     for l, count in convs:
         ms = float(np.mean([a.elapsed_time(b) for a, b in per[l.name]]))
         shapes.append({"layer": l.name, "count": count, "M": l.M(B), "N": l.C_out, "K": l.K,
-                       "engine": binding.bcnn_auto_engine(B, l.H, l.W, l.C_in, l.C_out, 1, 1, 1, 0),
-                       "ms_per_launch": ms, "tops": l.ops(B) / (ms / 1e3) / 1e12,
-                       "gbs": (l.in_bytes(B) + l.out_bits_bytes(B)) / (ms / 1e3) / 1e9})
+                       "engine": ("tc_ws" if l.C_out <= 128 and l.K >= 64 else "tc_i8") if module
+                       else binding.bcnn_auto_engine(B, l.H, l.W, l.C_in, l.C_out, 1, 1, 1, 0),
+                       "ms_per_launch": ms, "tops": l.ops(B) / (ms / 1e3) / 1e12})
+        # algorithmic bytes: packed input + packed output (+ fp16 identity read and fp16 map written by the module)
+        nbytes = l.in_bytes(B) + l.out_bits_bytes(B) + (4 * l.M(B) * l.C_out if module else 0)
+        shapes[-1].update({"gbs": nbytes / (ms / 1e3) / 1e9, "hbm_frac": nbytes / (ms / 1e3) / 1e9 / peaks["hbm_gbs"]})
     err = binding.bcnn_device_error()
     ops = 2 * sum(n * l.macs(B) for l, n in convs)
     print(json.dumps({
-        "mode": "paper1x1", "metric": "binary conv throughput (2*M*N*K bit-ops/s), the paper's 1x1 convolutions (Table 1)",
+        "mode": "paper1x1", "epilogue": args.epilogue, "metric": "binary conv throughput (2*M*N*K bit-ops/s), the paper's 1x1 convolutions (Table 1)",
         "value": ops / (ms_step / 1e3) / 1e12, "unit": UNIT, "ms_per_step": ms_step, "images_per_s": B / (ms_step / 1e3),
         "binary_macs_per_image": ops // (2 * B), "n_gpus": 1, "steps": args.steps, "data": "synthetic",
-        "config": {"workload": f"Table 1 network, binary 1x1 convolutions only, P = {P}, batch {B}", "launches": len(jobs),
+        "hbm_peak_gbs": peaks["hbm_gbs"], "peak_source": peaks["source"],
+        "config": {"workload": f"Table 1 network, binary 1x1 convolutions only, P = {P}, batch {B}, epilogue {args.epilogue}",
+                   "launches": len(jobs),
                    "launch": "CUDA graph replay"},
         "per_shape": shapes, "device_error": err}))
     return 0 if err == 0 else 1
@@ -563,6 +586,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--batch", type=int, default=256, help="paper1x1 mode: images per step")
+    ap.add_argument("--epilogue", default="threshold", choices=["threshold", "module"],
+                    help="paper1x1 mode: integer threshold, or the full convolution module (batch norm, fp16 identity, PReLU, next sign)")
     ap.add_argument("--branches", type=int, default=1, choices=[1, 2], help="paper1x1 mode: parallel binary branches P")
     args = ap.parse_args()
     if args.impl == "reference":

@@ -115,6 +115,25 @@ int bcnn_conv2d_b1_fused(const void *x_bits, const void *w_bits, const int32_t *
                          int kh, int kw, int stride, int pad, void *stream);
 
 /*
+ * Binary convolution followed by the rest of the paper's convolution module (Section 4.2.1, Figure 4: learnable
+ * bias -> sign -> binary conv -> batch norm -> + module identity -> PReLU; the bias + sign at the front is the
+ * producer of x_bits, the bias + sign of the NEXT module is emitted here), in one pass:
+ *   acc = the convolution's integer result (as bcnn_conv2d_b1)
+ *   t = acc * bn_scale[co] + bn_shift[co];  u = t + identity;  r = (u >= 0) ? u : prelu_slope[co] * u
+ *   y_real = fp16(r);   y bit = (y_real + next_bias[co] >= 0)
+ * Every step is one fp32 operation rounded to nearest even (no fused multiply-add); the sign is taken of the
+ * stored fp16 value, so it equals bcnn_pack applied to y_real.
+ *   bn_scale, bn_shift, prelu_slope  device fp32 [C_out];  next_bias device fp32 [C_out] or NULL (= 0)
+ *   identity  device fp16 NHWC [B][OH][OW][C_out] (the module's real input; needs the output's shape), or NULL
+ *   y_real    device fp16 NHWC [B][OH][OW][C_out];  y_bits device packed NHWC [B][OH][OW][C_out], or NULL
+ *   C_out % 32 == 0.  identity and y_real may be the same buffer (each element is read before it is written).
+ */
+int bcnn_conv2d_b1_module(const void *x_bits, const void *w_bits, const float *bn_scale, const float *bn_shift,
+                          const void *identity, const float *prelu_slope, const float *next_bias,
+                          void *y_real, void *y_bits, int B, int H, int W, int C_in, int C_out,
+                          int kh, int kw, int stride, int pad, void *stream);
+
+/*
  * Fused stem: bcnn_pack followed by the first binary 1x1 convolution with its threshold epilogue, without
  * writing the packed sign tensor in between (Section 4.1: the stem uses the same block, so even the first
  * convolution is binary; Table 1 "stem replicate": 4 real channels replicated 8x to 32 sign channels;

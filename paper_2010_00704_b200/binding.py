@@ -20,7 +20,7 @@ ENGINES = {"auto": ENGINE_AUTO, "lop3": ENGINE_LOP3, "mma_b1": ENGINE_MMA_B1, "t
            "mma_s8": ENGINE_MMA_S8, "tc_ws": ENGINE_TC_WS}
 
 EXPORTS = (
-    "bcnn_pack", "bcnn_stem_fused", "bcnn_gemm_b1", "bcnn_gemm_b1_fused", "bcnn_conv2d_b1", "bcnn_conv2d_b1_fused",
+    "bcnn_pack", "bcnn_stem_fused", "bcnn_gemm_b1", "bcnn_gemm_b1_fused", "bcnn_conv2d_b1", "bcnn_conv2d_b1_fused", "bcnn_conv2d_b1_module",
     "bcnn_conv2d_b1_engine", "bcnn_gemm_b1_engine", "bcnn_auto_engine", "bcnn_device_error", "bcnn_status_string",
     "bcnn_version",
 )
@@ -48,6 +48,7 @@ def load() -> ctypes.CDLL:
         lib.bcnn_gemm_b1_fused.argtypes = [vp, vp, vp, vp, i64, i32, i32, vp]
         lib.bcnn_conv2d_b1.argtypes = [vp, vp, vp] + [i32] * 9 + [vp]
         lib.bcnn_conv2d_b1_fused.argtypes = [vp, vp, vp, vp] + [i32] * 9 + [vp]
+        lib.bcnn_conv2d_b1_module.argtypes = [vp] * 9 + [i32] * 9 + [vp]
         lib.bcnn_conv2d_b1_engine.argtypes = [i32, vp, vp, vp, vp] + [i32] * 9 + [vp]
         lib.bcnn_gemm_b1_engine.argtypes = [i32, vp, vp, vp, vp, i64, i32, i32, vp]
         lib.bcnn_auto_engine.argtypes = [i32] * 10
@@ -128,6 +129,15 @@ def bcnn_conv2d_b1_fused(x_bits, w_bits, thr, y_bits, B, H, W, C_in, C_out, kh, 
     _check(load().bcnn_conv2d_b1_engine(engine, _p(x_bits), _p(w_bits), _p(thr), _p(y_bits), B, H, W, C_in,
                                         C_out, kh, kw, stride, pad, _stream()), "bcnn_conv2d_b1_fused")
     return y_bits
+
+
+def bcnn_conv2d_b1_module(x_bits, w_bits, bn_scale, bn_shift, identity, prelu_slope, next_bias, y_real, y_bits,
+                          B, H, W, C_in, C_out, kh, kw, stride, pad):
+    """Binary conv -> batch norm -> + identity (fp16) -> PReLU -> fp16 map and the next module's packed signs."""
+    _check(load().bcnn_conv2d_b1_module(_p(x_bits), _p(w_bits), _p(bn_scale), _p(bn_shift), _p(identity),
+                                        _p(prelu_slope), _p(next_bias), _p(y_real), _p(y_bits), B, H, W, C_in, C_out,
+                                        kh, kw, stride, pad, _stream()), "bcnn_conv2d_b1_module")
+    return y_real, y_bits
 
 
 def bcnn_auto_engine(B, H, W, C_in, C_out, kh, kw, stride, pad, fused=True) -> str:

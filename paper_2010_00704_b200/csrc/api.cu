@@ -63,6 +63,10 @@ int make_conv_problem(ConvProblem &p, const void *x, const void *w, const int32_
     p.M = (int)M;
     p.cw_magic = p.cw == 1 ? 0u : (uint32_t)((1ULL << 32) / (uint64_t)p.cw) + 1u;
     p.err = nullptr;
+    p.mode = fused ? 1 : 0;
+    p.bn_scale = p.bn_shift = p.slope = p.next_bias = nullptr;
+    p.identity = nullptr;
+    p.y_real = nullptr;
     exact_div_params((uint32_t)OW, p.ow_mul, p.ow_shift);
     exact_div_params((uint32_t)(OH * OW), p.ohw_mul, p.ohw_shift);
     p.kw_magic = kw == 1 ? 0u : (uint32_t)((1ULL << 32) / (uint64_t)kw) + 1u;
@@ -175,6 +179,33 @@ int bcnn_conv2d_b1_fused(const void *x_bits, const void *w_bits, const int32_t *
     if (!thr) return BCNN_ERR_INVALID_ARG;
     return bcnn_conv2d_b1_engine(BCNN_ENGINE_AUTO, x_bits, w_bits, thr, y_bits, B, H, W, C_in, C_out,
                                  kh, kw, stride, pad, stream);
+}
+
+int bcnn_conv2d_b1_module(const void *x_bits, const void *w_bits, const float *bn_scale, const float *bn_shift,
+                          const void *identity, const float *prelu_slope, const float *next_bias,
+                          void *y_real, void *y_bits, int B, int H, int W, int C_in, int C_out,
+                          int kh, int kw, int stride, int pad, void *stream)
+{
+    if (!bn_scale || !bn_shift || !prelu_slope || !y_real) return BCNN_ERR_INVALID_ARG;
+    ConvProblem p;
+    // validated like the int32 convolution whose result it post-processes (y_real stands in for the output)
+    const int st = make_conv_problem(p, x_bits, w_bits, nullptr, y_real, B, H, W, C_in, C_out, kh, kw, stride, pad, false);
+    if (st != BCNN_OK) return st;
+    if (C_out % 32 != 0) return BCNN_ERR_UNSUPPORTED;
+    if (!aligned16(bn_scale) || !aligned16(bn_shift) || !aligned16(prelu_slope) || (next_bias && !aligned16(next_bias)) ||
+        (identity && !aligned16(identity)) || (y_bits && !aligned16(y_bits)))
+        return BCNN_ERR_ALIGNMENT;
+    p.mode = 2;
+    p.bn_scale = bn_scale;
+    p.bn_shift = bn_shift;
+    p.slope = prelu_slope;
+    p.next_bias = next_bias;
+    p.identity = static_cast<const uint16_t *>(identity);
+    p.y_real = static_cast<uint16_t *>(y_real);
+    p.out = y_bits;
+    // the two tcgen05 engines carry this epilogue
+    if (p.C_out <= 128 && p.K >= 64 && conv_tc_ws_supports(p)) return launch_conv_tc_ws(p, static_cast<cudaStream_t>(stream));
+    return launch_conv_tc_i8(p, static_cast<cudaStream_t>(stream));
 }
 
 int bcnn_conv2d_b1_engine(int engine, const void *x_bits, const void *w_bits, const int32_t *thr, void *out,

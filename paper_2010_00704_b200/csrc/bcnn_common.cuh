@@ -22,6 +22,11 @@ struct ConvProblem {
     uint32_t cw_magic;   // floor(2^32 / cw) + 1 (0 when cw == 1): n / cw == umulhi(n, magic) for n*cw < 2^32
     uint32_t kw_magic;   // same for the kernel width kw
     int *err;            // device error word (bounded waits report here)
+    // convolution-module epilogue (mode == 2): batch norm scale / shift, fp16 identity, PReLU slope, next bias
+    int mode;            // 0: int32 output, 1: integer threshold -> packed bits, 2: module epilogue
+    const float *bn_scale, *bn_shift, *slope, *next_bias;   // [C_out]; next_bias may be nullptr (0)
+    const uint16_t *identity;                               // fp16 [M][C_out] or nullptr
+    uint16_t *y_real;                                       // fp16 [M][C_out]; the packed next signs go to `out` (may be nullptr)
     uint32_t ow_mul, ow_shift;    // exact division of any 32-bit value by OW      (see exact_div)
     uint32_t ohw_mul, ohw_shift;  // exact division of any 32-bit value by OH * OW
 };

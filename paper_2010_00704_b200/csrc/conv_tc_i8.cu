@@ -63,11 +63,12 @@ __host__ __device__ inline int smem_bytes(int ktab_words)
     return 1024 + C::STAGES * C::W_BYTES + C::BITS_BYTES + C::CONST_BYTES + ktab_words * 4;
 }
 
-template <int BN, bool FUSED>
+template <int BN, int MODE>
 __global__ void __launch_bounds__(Cfg<BN>::THREADS, 1)
 conv_tc_i8_kernel(const ConvProblem p, const int ktab_words)
 {
     using C = Cfg<BN>;
+    constexpr bool FUSED = MODE == 1, MODULE = MODE == 2;
     constexpr int NBUF = C::NBUF;
     constexpr int STAGES = C::STAGES;
     constexpr int SLOTS = C::SLOTS;
@@ -225,6 +226,21 @@ conv_tc_i8_kernel(const ConvProblem p, const int ktab_words)
                             acc = __funnelshift_l((uint32_t)((int)v[4 * i4 + 0] + rowc + (int)cc.x), acc, 1);
                         }
                         words[ch] = ~acc;
+                    } else if (MODULE) {
+                        int dot[32];
+#pragma unroll
+                        for (int i4 = 0; i4 < 8; ++i4) {
+                            uint4 cc = ld_shared_v4(c0_addr + 4u * (col0 + 4 * i4));
+                            if (two) {
+                                const uint4 c2 = ld_shared_v4(c1_addr + 4u * (col0 + 4 * i4));
+                                cc.x += c2.x; cc.y += c2.y; cc.z += c2.z; cc.w += c2.w;
+                            }
+                            dot[4 * i4 + 0] = (int)(v[4 * i4 + 0] >> 5) + rowc + (int)cc.x;
+                            dot[4 * i4 + 1] = (int)(v[4 * i4 + 1] >> 5) + rowc + (int)cc.y;
+                            dot[4 * i4 + 2] = (int)(v[4 * i4 + 2] >> 5) + rowc + (int)cc.z;
+                            dot[4 * i4 + 3] = (int)(v[4 * i4 + 3] >> 5) + rowc + (int)cc.w;
+                        }
+                        words[ch] = module_chunk(p, dot, em, n0 + col0, em < p.M);
                     } else if (em < p.M) {
                         int32_t *dst = static_cast<int32_t *>(p.out) + (long)em * p.C_out + n0 + col0;
                         const bool vec = (p.C_out & 3) == 0 && (n0 + col0 + 32 <= p.C_out);
@@ -258,7 +274,7 @@ conv_tc_i8_kernel(const ConvProblem p, const int ktab_words)
             __syncwarp();
             if (lane == 0) mbar_arrive(tempty_bar(buf));
             if (++buf == NBUF) { buf = 0; buf_phase ^= 1u; }
-            if (FUSED && em < p.M) {
+            if ((FUSED || (MODULE && p.out != nullptr)) && em < p.M) {
                 const int owords = p.C_out >> 5;
                 uint32_t *dst = static_cast<uint32_t *>(p.out) + (long)em * owords + (n0 >> 5);
                 if ((owords & 3) == 0 && n0 + BN <= p.C_out) {
@@ -446,7 +462,7 @@ int launch_bn(const ConvProblem &p0, cudaStream_t stream)
     const unsigned grid = (unsigned)(total < sms ? total : sms);
     const int ktw = ktab_words_for(p);
     const int smem = smem_bytes<BN>(ktw);
-    void (*k)(const ConvProblem, const int) = p.thr ? conv_tc_i8_kernel<BN, true> : conv_tc_i8_kernel<BN, false>;
+    void (*k)(const ConvProblem, const int) = p.mode == 2 ? conv_tc_i8_kernel<BN, 2> : (p.mode == 1 ? conv_tc_i8_kernel<BN, 1> : conv_tc_i8_kernel<BN, 0>);
     // the attribute is a property of the kernel, not of the launch: always the limit, so that a captured
     // launch stays valid whatever later calls with other shapes ask for
     if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, MAX_SMEM) != cudaSuccess) return BCNN_ERR_CUDA;
@@ -458,7 +474,7 @@ int launch_bn(const ConvProblem &p0, cudaStream_t stream)
 
 bool conv_tc_i8_supports(const ConvProblem &p)
 {
-    if (p.thr != nullptr && (p.C_out % 32 != 0)) return false;
+    if (p.mode != 0 && (p.C_out % 32 != 0)) return false;
     if (p.kh * p.kw > 31) return false;                       // one validity bit per tap
     if ((long)p.B * p.H * p.W * p.cw >= (1L << 31)) return false;     // rows address the input by 32-bit word offsets
     if (smem_bytes<256>(ktab_words_for(p)) > MAX_SMEM) return false;   // the K-word table of the gather must fit

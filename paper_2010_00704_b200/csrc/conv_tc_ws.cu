@@ -90,11 +90,12 @@ __host__ __device__ inline WsLayout ws_layout(int kwords)
     return l;
 }
 
-template <int BN, int G, bool DUAL, bool FUSED>
+template <int BN, int G, bool DUAL, int MODE>
 __global__ void __launch_bounds__(Cfg<BN, G, DUAL>::BOUND_THREADS, Cfg<BN, G, DUAL>::CTAS_PER_SM)
 conv_tc_ws_kernel(const ConvProblem p)
 {
     using C = Cfg<BN, G, DUAL>;
+    constexpr bool FUSED = MODE == 1, MODULE = MODE == 2;
     constexpr int BNX = C::BNX;
     constexpr int NBUF = C::NBUF;
     constexpr int MAX_STAGES = 8;
@@ -269,6 +270,17 @@ conv_tc_ws_kernel(const ConvProblem p)
                             acc = __funnelshift_l((uint32_t)((int)v[4 * i4 + 0] + (int)cc.x), acc, 1);
                         }
                         words[ch] = ~acc;
+                    } else if (MODULE) {
+                        int dot[32];
+#pragma unroll
+                        for (int i4 = 0; i4 < 8; ++i4) {
+                            const uint4 cc = ld_shared_v4(colc_addr + 4u * (col0 + 4 * i4));
+                            dot[4 * i4 + 0] = ((int)v[4 * i4 + 0] >> 5) + (int)cc.x;
+                            dot[4 * i4 + 1] = ((int)v[4 * i4 + 1] >> 5) + (int)cc.y;
+                            dot[4 * i4 + 2] = ((int)v[4 * i4 + 2] >> 5) + (int)cc.z;
+                            dot[4 * i4 + 3] = ((int)v[4 * i4 + 3] >> 5) + (int)cc.w;
+                        }
+                        words[ch] = module_chunk(p, dot, em, col0, em < p.M);
                     } else if (em < p.M) {
                         int32_t *dst = static_cast<int32_t *>(p.out) + (long)em * p.C_out + col0;
                         const bool vec = (p.C_out & 3) == 0 && (col0 + 32 <= p.C_out);
@@ -297,7 +309,7 @@ conv_tc_ws_kernel(const ConvProblem p)
             __syncwarp();
             if (lane == 0) mbar_arrive(tempty_bar(buf));
             if (++buf == NBUF) { buf = 0; buf_phase ^= 1u; }
-            if (FUSED && em < p.M) {
+            if ((FUSED || (MODULE && p.out != nullptr)) && em < p.M) {
                 const int owords = p.C_out >> 5;
                 uint32_t *dst = static_cast<uint32_t *>(p.out) + (long)em * owords;
                 if (BN == 128 && owords == 4) {
@@ -481,7 +493,7 @@ int launch_ws(const ConvProblem &p0, cudaStream_t stream)
     const long m_tiles = ((long)p.M + BM - 1) / BM;
     const long slots = (long)sms * C::CTAS_PER_SM;
     const unsigned grid = (unsigned)(m_tiles < slots ? m_tiles : slots);
-    void (*k)(const ConvProblem) = p.thr ? conv_tc_ws_kernel<BN, G, DUAL, true> : conv_tc_ws_kernel<BN, G, DUAL, false>;
+    void (*k)(const ConvProblem) = p.mode == 2 ? conv_tc_ws_kernel<BN, G, DUAL, 2> : (p.mode == 1 ? conv_tc_ws_kernel<BN, G, DUAL, 1> : conv_tc_ws_kernel<BN, G, DUAL, 0>);
     // the attribute is a property of the kernel, not of the launch: always the configuration's limit, so
     // that a captured launch stays valid whatever later calls with other shapes ask for
     if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, DUAL ? 113 * 1024 : MAX_SMEM - 1024) != cudaSuccess) return BCNN_ERR_CUDA;
@@ -501,7 +513,7 @@ bool fits(const ConvProblem &p)
 
 bool conv_tc_ws_supports(const ConvProblem &p)
 {
-    if (p.thr != nullptr && (p.C_out % 32 != 0)) return false;
+    if (p.mode != 0 && (p.C_out % 32 != 0)) return false;
     if (p.C_out > 128 || p.kh * p.kw > 31 || p.K > (1 << 16)) return false;
     // rows address the input by 32-bit word offsets
     if ((long)p.B * p.H * p.W * p.cw >= (1L << 31)) return false;

@@ -3,6 +3,7 @@
 // cp.async staging, shared-memory descriptors and the bit -> byte expansions.
 #pragma once
 #include "bcnn_common.cuh"
+#include <cuda_fp16.h>
 
 namespace bcnn {
 namespace tc {
@@ -389,6 +390,54 @@ __device__ __forceinline__ void gather_stage(const uint32_t *x, const RowCursor 
         const int idx = ok ? rc.base + (int)ent[2 * u] : 0;
         cp_async_zfill<GW * 4>(dst + (uint32_t)(u * GW * 4), x + idx, ok ? (uint32_t)(GW * 4) : 0u);
     }
+}
+
+// Convolution-module epilogue (Section 4.2.1) for 32 consecutive output channels n0 .. n0+31 of one output row:
+//   t = dot * scale + shift;  u = t + identity;  r = u >= 0 ? u : slope * u;  y = fp16(r);  bit = (y + next_bias >= 0)
+// one fp32 operation per step, each rounded to nearest (no fused multiply-add), the sign taken of the stored
+// fp16 value.  Stores the 32 fp16 values (when `live`) and returns the 32 sign bits (bit i = channel n0 + i).
+// The channel count is a multiple of 32, so every 8-channel group is 16-byte aligned.
+__device__ __forceinline__ uint32_t module_chunk(const ConvProblem &p, const int (&dot)[32], long row, int n0, bool live)
+{
+    uint32_t bits = 0;
+    const long base = row * p.C_out + n0;
+#pragma unroll
+    for (int g = 0; g < 4; ++g) {                           // 8 channels per group
+        uint4 idv = make_uint4(0u, 0u, 0u, 0u);
+        if (p.identity && live) idv = __ldg(reinterpret_cast<const uint4 *>(p.identity + base + 8 * g));
+        const uint32_t idw[4] = {idv.x, idv.y, idv.z, idv.w};
+        uint32_t ow[4];
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+            const int n = n0 + 8 * g + 4 * h;
+            const float4 sc = __ldg(reinterpret_cast<const float4 *>(p.bn_scale + n));
+            const float4 sh = __ldg(reinterpret_cast<const float4 *>(p.bn_shift + n));
+            const float4 sl = __ldg(reinterpret_cast<const float4 *>(p.slope + n));
+            float4 nb = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (p.next_bias) nb = __ldg(reinterpret_cast<const float4 *>(p.next_bias + n));
+            const float scs[4] = {sc.x, sc.y, sc.z, sc.w}, shs[4] = {sh.x, sh.y, sh.z, sh.w};
+            const float sls[4] = {sl.x, sl.y, sl.z, sl.w}, nbs[4] = {nb.x, nb.y, nb.z, nb.w};
+            unsigned short hv[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const int c = 8 * g + 4 * h + e;
+                const uint32_t pair = idw[2 * h + (e >> 1)];
+                const __half idh = __ushort_as_half((unsigned short)((e & 1) ? (pair >> 16) : (pair & 0xFFFFu)));
+                float t = __fmul_rn(__int2float_rn(dot[c]), scs[e]);
+                t = __fadd_rn(t, shs[e]);
+                const float u = p.identity ? __fadd_rn(t, __half2float(idh)) : t;
+                const float r = (u >= 0.0f) ? u : __fmul_rn(sls[e], u);
+                const __half y = __float2half_rn(r);
+                hv[e] = __half_as_ushort(y);
+                const float sv = __fadd_rn(__half2float(y), nbs[e]);
+                bits |= (sv >= 0.0f ? 1u : 0u) << c;
+            }
+            ow[2 * h] = (uint32_t)hv[0] | ((uint32_t)hv[1] << 16);
+            ow[2 * h + 1] = (uint32_t)hv[2] | ((uint32_t)hv[3] << 16);
+        }
+        if (live) *reinterpret_cast<uint4 *>(p.y_real + base + 8 * g) = make_uint4(ow[0], ow[1], ow[2], ow[3]);
+    }
+    return bits;
 }
 
 }  // namespace tc

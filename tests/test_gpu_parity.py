@@ -291,3 +291,77 @@ def test_errors_launch_nothing(bk):
     torch.cuda.synchronize()
     assert int(a.sum()) == 0
     assert bk.bcnn_device_error() == 0
+
+
+MODULE_SHAPES = [
+    # B, H, W, Ci, Co, k, stride, pad
+    (2, 9, 13, 64, 64, 1, 1, 0),       # weight-stationary engine, the paper's 1x1 module shape
+    (1, 20, 20, 128, 128, 1, 1, 0),
+    (2, 12, 10, 64, 96, 3, 2, 1),      # 3x3 stride 2, ragged N tile
+    (3, 7, 11, 32, 32, 1, 1, 0),       # one-word K: streaming engine
+    (1, 14, 14, 256, 256, 1, 1, 0),    # streaming engine, 256-wide tile
+    (2, 7, 7, 512, 1024, 1, 1, 0),     # several N tiles
+    (1, 10, 10, 128, 320, 3, 1, 1),    # ragged N tile of the streaming engine, K = 1152
+]
+
+
+@pytest.mark.parametrize("variant", ["full", "no_identity", "no_bits", "in_place"])
+@pytest.mark.parametrize("shape", MODULE_SHAPES)
+def test_conv_module(bk, oracle, shape, variant):
+    # binary conv -> batch norm -> + identity -> PReLU -> fp16 map + next signs, bit for bit against the oracle
+    B, H, W, Ci, Co, k, stride, pad = shape
+    rng = np.random.default_rng(7000 + sum(shape))
+    x, w = synth.pm1(rng, (B, H, W, Ci)), synth.pm1(rng, (Co, k, k, Ci))
+    K = k * k * Ci
+    scale = (rng.standard_normal(Co) / np.sqrt(K)).astype(np.float32)
+    scale[::7] *= -1                                       # negative batch-norm scales need no folding here
+    shift = rng.standard_normal(Co).astype(np.float32)
+    slope = rng.uniform(-0.25, 1.0, Co).astype(np.float32)
+    nbias = rng.standard_normal(Co).astype(np.float32)
+    OH, OW = bk.out_hw(H, W, k, k, stride, pad)
+    ident = rng.standard_normal((B, OH, OW, Co)).astype(np.float16)
+    acc = oracle.conv2d(x, w, stride, pad)
+    # plant exact zeros and sign ties: channel 0 passes acc through and its next bias cancels a value that occurs
+    scale[0], shift[0], slope[0] = 1.0, 0.0, 1.0
+    ident[..., 0] = 0
+    nbias[0] = -float(acc[0, 0, 0, 0])
+    has_id = variant != "no_identity"
+    has_bits = variant != "no_bits"
+    want_y, want_s = oracle.conv_module(acc, scale, shift, ident if has_id else None, slope, nbias if has_bits else None)
+    n = B * OH * OW * Co
+    raw_y, ybuf = guard_alloc(2 * n)
+    raw_b, bbuf = guard_alloc(n // 8)
+    id_dev = None
+    if has_id:
+        if variant == "in_place":
+            ybuf.copy_(dev(ident.view(np.uint8).reshape(-1)))
+            id_dev = ybuf
+        else:
+            id_dev = dev(ident.view(np.uint8).reshape(-1))
+    bk.bcnn_conv2d_b1_module(dev(synth.pack_bits(x)), dev(synth.pack_bits(w)), dev(scale), dev(shift), id_dev, dev(slope),
+                             dev(nbias) if has_bits else None, ybuf, bbuf if has_bits else None,
+                             B, H, W, Ci, Co, k, k, stride, pad)
+    torch.cuda.synchronize()
+    check_guards(raw_y, 2 * n)
+    check_guards(raw_b, n // 8)
+    got_y = ybuf.cpu().numpy().view(np.uint16).reshape(B, OH, OW, Co)
+    assert np.array_equal(got_y, want_y.view(np.uint16))
+    if has_bits:
+        assert np.array_equal(synth.unpack_bits(bbuf.cpu().numpy().reshape(B, OH, OW, Co // 8)), want_s)
+    assert bk.bcnn_device_error() == 0
+
+
+def test_conv_module_errors(bk):
+    a = torch.zeros(1 << 16, dtype=torch.uint8, device="cuda")
+    f = torch.zeros(1024, dtype=torch.float32, device="cuda")
+    with pytest.raises(bk.BcnnError) as e:
+        bk.bcnn_conv2d_b1_module(a, a, f, f, None, f, None, a, None, 1, 4, 4, 32, 48, 1, 1, 1, 0)   # C_out % 32 != 0
+    assert e.value.status == -2
+    with pytest.raises(bk.BcnnError) as e:
+        bk.bcnn_conv2d_b1_module(a, a, None, f, None, f, None, a, None, 1, 4, 4, 32, 32, 1, 1, 1, 0)
+    assert e.value.status == -1
+    with pytest.raises(bk.BcnnError) as e:
+        bk.bcnn_conv2d_b1_module(a, a, f[1:], f, None, f, None, a, None, 1, 4, 4, 32, 32, 1, 1, 1, 0)
+    assert e.value.status == -3
+    torch.cuda.synchronize()
+    assert int(a.sum()) == 0
