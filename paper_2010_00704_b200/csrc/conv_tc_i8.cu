@@ -57,10 +57,11 @@ template <int BN> struct Cfg {
 };
 
 template <int BN>
-__host__ __device__ inline int smem_bytes(int ktab_words)
+__host__ __device__ inline int smem_bytes(int ktab_words, bool module = false)
 {
     using C = Cfg<BN>;
-    return 1024 + C::STAGES * C::W_BYTES + C::BITS_BYTES + C::CONST_BYTES + ktab_words * 4;
+    // module epilogue: + the identity staging ring
+    return 1024 + C::STAGES * C::W_BYTES + C::BITS_BYTES + C::CONST_BYTES + ktab_words * 4 + (module ? ID_RING_BYTES + 16 : 0);
 }
 
 template <int BN, int MODE>
@@ -91,6 +92,7 @@ conv_tc_i8_kernel(const ConvProblem p, const int ktab_words)
     const uint32_t bits_ring = wring + STAGES * C::W_BYTES;               // [PF][PROD_THREADS][16 B]
     const uint32_t consts = bits_ring + C::BITS_BYTES;                    // [SLOTS][G][BM + BN] int32
     const uint32_t ktab_addr = consts + C::CONST_BYTES;                   // unit table of the gather: {word offset, tap bit}
+    const uint32_t idring = (ktab_addr + (uint32_t)ktab_words * 4u + 15u) & ~15u;   // module epilogue only: [ID_SLOTS][BM rows][80 B]
     const uint32_t bar0 = smem_u32(bars);
     auto full_bar = [&](int s) { return bar0 + 8u * s; };
     auto empty_bar = [&](int s) { return bar0 + 8u * (8 + s); };
@@ -180,6 +182,28 @@ conv_tc_i8_kernel(const ConvProblem p, const int ktab_words)
         bool alive = true;
         int buf = 0;
         uint32_t buf_phase = 0;
+        // module epilogue: the identity values of this thread's row are staged ID_AHEAD live chunks ahead (a chunk is
+        // live when its first channel exists), in ring slot (live chunk number) % ID_SLOTS
+        const uint32_t id_row = idring + (uint32_t)erow * ID_ROW_BYTES;
+        int pf_ti = 0, pf_ch = 0, pf_slot = 0, cur_slot = 0;
+        auto prefetch_next = [&]() {
+            bool queued = false;
+            while (pf_ti < my_tiles && !queued) {
+                const int t = (int)blockIdx.x + pf_ti * (int)gridDim.x;
+                const int nt = t / m_tiles, mt = t - nt * m_tiles;
+                const int n = nt * BN + pf_ch * 32;
+                if (n < p.C_out) {
+                    const long row = (long)mt * BM + erow;
+                    module_prefetch(p, id_row + (uint32_t)pf_slot * (BM * ID_ROW_BYTES), row, n, row < p.M);
+                    queued = true;
+                }
+                if (++pf_ch == BN / 32) { pf_ch = 0; ++pf_ti; }
+            }
+            if (!queued) cp_async_commit();
+            if (++pf_slot == ID_SLOTS) pf_slot = 0;
+        };
+        if (MODULE)
+            for (int a = 0; a < ID_AHEAD; ++a) prefetch_next();
         for (int ti = 0; ti < my_tiles; ++ti) {
             const int tile = (int)blockIdx.x + ti * (int)gridDim.x;
             const int n_tile = tile / m_tiles, m_tile = tile - n_tile * m_tiles;
@@ -240,7 +264,10 @@ conv_tc_i8_kernel(const ConvProblem p, const int ktab_words)
                             dot[4 * i4 + 2] = (int)(v[4 * i4 + 2] >> 5) + rowc + (int)cc.z;
                             dot[4 * i4 + 3] = (int)(v[4 * i4 + 3] >> 5) + rowc + (int)cc.w;
                         }
-                        words[ch] = module_chunk(p, dot, em, n0 + col0, em < p.M);
+                        prefetch_next();
+                        cp_async_wait<ID_AHEAD>();                    // this chunk's copy has landed
+                        words[ch] = module_chunk(p, dot, id_row + (uint32_t)cur_slot * (BM * ID_ROW_BYTES), em, n0 + col0, em < p.M);
+                        if (++cur_slot == ID_SLOTS) cur_slot = 0;
                     } else if (em < p.M) {
                         int32_t *dst = static_cast<int32_t *>(p.out) + (long)em * p.C_out + n0 + col0;
                         const bool vec = (p.C_out & 3) == 0 && (n0 + col0 + 32 <= p.C_out);
@@ -289,6 +316,7 @@ conv_tc_i8_kernel(const ConvProblem p, const int ktab_words)
                 }
             }
         }
+        if (MODULE) cp_async_wait<0>();
     } else {
         // ------------------------------------------------------------------ producers
         const int pw = warp - C::FIRST_PRODUCER_WARP;            // producer warp index
@@ -461,7 +489,8 @@ int launch_bn(const ConvProblem &p0, cudaStream_t stream)
     if (total >= (1L << 31)) return BCNN_ERR_UNSUPPORTED;
     const unsigned grid = (unsigned)(total < sms ? total : sms);
     const int ktw = ktab_words_for(p);
-    const int smem = smem_bytes<BN>(ktw);
+    const int smem = smem_bytes<BN>(ktw, p.mode == 2);
+    if (smem > MAX_SMEM) return BCNN_ERR_UNSUPPORTED;
     void (*k)(const ConvProblem, const int) = p.mode == 2 ? conv_tc_i8_kernel<BN, 2> : (p.mode == 1 ? conv_tc_i8_kernel<BN, 1> : conv_tc_i8_kernel<BN, 0>);
     // the attribute is a property of the kernel, not of the launch: always the limit, so that a captured
     // launch stays valid whatever later calls with other shapes ask for
@@ -487,7 +516,8 @@ int launch_conv_tc_i8(const ConvProblem &p, cudaStream_t stream)
     if (!conv_tc_i8_supports(p)) return BCNN_ERR_UNSUPPORTED;
     // 256-wide tiles have a single accumulator buffer (tensor memory also holds the activation
     // ring), so their epilogue is not overlapped: worth it only when the K loop is long
-    if (p.C_out > 128 && p.kwords >= 24) return launch_bn<256>(p, stream);
+    // (the module epilogue's staging ring only fits beside the 128-wide tiles' weight ring)
+    if (p.C_out > 128 && p.kwords >= 24 && p.mode != 2) return launch_bn<256>(p, stream);
     return launch_bn<128>(p, stream);
 }
 

@@ -70,7 +70,7 @@ struct WsLayout {
 };
 
 template <int BN, int G, bool DUAL>
-__host__ __device__ inline WsLayout ws_layout(int kwords)
+__host__ __device__ inline WsLayout ws_layout(int kwords, bool module)
 {
     using C = Cfg<BN, G, DUAL>;
     WsLayout l;
@@ -82,6 +82,7 @@ __host__ __device__ inline WsLayout ws_layout(int kwords)
     l.row_kt = (l.ktiles <= 3 && C::STAGES >= (G - 1) * l.ktiles + 1) ? l.ktiles : 0;
     l.bits_bytes = C::BITS_BYTES * (l.row_kt ? l.row_kt : 1);
     l.smem = 1024 + l.ktiles * C::W_TILE_BYTES + l.bits_bytes + BN * 4 + l.ktiles * 32;
+    if (module) l.smem += ID_RING_BYTES + 16;                 // identity staging ring of the module epilogue
     // Tensor memory is shared out by the resident CTAs (all 512 columns, or 256 each for two): ask
     // for enough shared memory that no further CTA of this kernel fits on the SM (it would sit in
     // tcgen05.alloc until a neighbour exits).
@@ -107,7 +108,7 @@ conv_tc_ws_kernel(const ConvProblem p)
 
     const int tid = threadIdx.x;
     const int warp = tid >> 5, lane = tid & 31;
-    const WsLayout L = ws_layout<BN, G, DUAL>(p.kwords);
+    const WsLayout L = ws_layout<BN, G, DUAL>(p.kwords, MODULE);
     const int ktiles = L.ktiles;
     constexpr int STAGES = C::STAGES;
     const int m_tiles = (p.M + BM - 1) / BM;
@@ -119,6 +120,7 @@ conv_tc_ws_kernel(const ConvProblem p)
     const uint32_t bits_ring = wexp + (uint32_t)ktiles * C::W_TILE_BYTES; // [PF][PROD_THREADS][16 B]
     const uint32_t colc_addr = bits_ring + (uint32_t)L.bits_bytes;                 // [BN] int32
     const uint32_t ktab_addr = colc_addr + BN * 4;                        // unit table: [ktiles * 4 / gw] x {word offset, tap bit}
+    const uint32_t idring = (ktab_addr + (uint32_t)ktiles * 32u + 15u) & ~15u;   // module epilogue only: [ID_SLOTS][BM rows][80 B]
     const uint32_t bar0 = smem_u32(bars);
     auto full_bar = [&](int s) { return bar0 + 8u * s; };
     auto empty_bar = [&](int s) { return bar0 + 8u * (MAX_STAGES + s); };
@@ -243,6 +245,23 @@ conv_tc_ws_kernel(const ConvProblem p)
         bool alive = true;
         int buf = 0;
         uint32_t buf_phase = 0;
+        // module epilogue: chunk q of this thread's row sequence = (tile q / nch, chunk q % nch); its identity values
+        // are staged ID_AHEAD chunks ahead in ring slot q % ID_SLOTS
+        const int nch = (p.C_out + 31) >> 5;
+        const uint32_t id_row = idring + (uint32_t)erow * ID_ROW_BYTES;
+        int pf_ti = 0, pf_ch = 0, pf_slot = 0, cur_slot = 0;
+        auto prefetch_next = [&]() {
+            if (pf_ti < my_tiles) {
+                const long row = (long)((int)blockIdx.x + pf_ti * (int)gridDim.x) * BM + erow;
+                module_prefetch(p, id_row + (uint32_t)pf_slot * (BM * ID_ROW_BYTES), row, pf_ch * 32, row < p.M);
+                if (++pf_ch == nch) { pf_ch = 0; ++pf_ti; }
+            } else {
+                cp_async_commit();
+            }
+            if (++pf_slot == ID_SLOTS) pf_slot = 0;
+        };
+        if (MODULE)
+            for (int a = 0; a < ID_AHEAD; ++a) prefetch_next();
         for (int ti = 0; ti < my_tiles; ++ti) {
             const int m_tile = (int)blockIdx.x + ti * (int)gridDim.x;
             const int em = m_tile * BM + erow;
@@ -280,7 +299,10 @@ conv_tc_ws_kernel(const ConvProblem p)
                             dot[4 * i4 + 2] = ((int)v[4 * i4 + 2] >> 5) + (int)cc.z;
                             dot[4 * i4 + 3] = ((int)v[4 * i4 + 3] >> 5) + (int)cc.w;
                         }
-                        words[ch] = module_chunk(p, dot, em, col0, em < p.M);
+                        prefetch_next();
+                        cp_async_wait<ID_AHEAD>();                    // this chunk's copy has landed
+                        words[ch] = module_chunk(p, dot, id_row + (uint32_t)cur_slot * (BM * ID_ROW_BYTES), em, col0, em < p.M);
+                        if (++cur_slot == ID_SLOTS) cur_slot = 0;
                     } else if (em < p.M) {
                         int32_t *dst = static_cast<int32_t *>(p.out) + (long)em * p.C_out + col0;
                         const bool vec = (p.C_out & 3) == 0 && (col0 + 32 <= p.C_out);
@@ -323,6 +345,7 @@ conv_tc_ws_kernel(const ConvProblem p)
                 }
             }
         }
+        if (MODULE) cp_async_wait<0>();
     } else {
         // ------------------------------------------------------------------ producers
         // Group g takes items g, g + G, ... of the CTA's flattened (tile, stage) list.  Per item a
@@ -489,7 +512,7 @@ int launch_ws(const ConvProblem &p0, cudaStream_t stream)
     cudaGetDevice(&dev);
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     using C = Cfg<BN, G, DUAL>;
-    const WsLayout L = ws_layout<BN, G, DUAL>(p.kwords);
+    const WsLayout L = ws_layout<BN, G, DUAL>(p.kwords, p.mode == 2);
     const long m_tiles = ((long)p.M + BM - 1) / BM;
     const long slots = (long)sms * C::CTAS_PER_SM;
     const unsigned grid = (unsigned)(m_tiles < slots ? m_tiles : slots);
@@ -506,7 +529,7 @@ int launch_ws(const ConvProblem &p0, cudaStream_t stream)
 template <int BN, int G, bool DUAL>
 bool fits(const ConvProblem &p)
 {
-    return ws_layout<BN, G, DUAL>(p.kwords).smem <= (DUAL ? 113 * 1024 : MAX_SMEM - 1024);
+    return ws_layout<BN, G, DUAL>(p.kwords, p.mode == 2).smem <= (DUAL ? 113 * 1024 : MAX_SMEM - 1024);
 }
 
 }  // namespace

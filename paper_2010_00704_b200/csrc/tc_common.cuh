@@ -392,19 +392,47 @@ __device__ __forceinline__ void gather_stage(const uint32_t *x, const RowCursor 
     }
 }
 
-// Convolution-module epilogue (Section 4.2.1) for 32 consecutive output channels n0 .. n0+31 of one output row:
+// Convolution-module epilogue (Section 4.2.1).
+//
+// Identity staging: an epilogue thread owns one output row and walks its 32-channel chunks in order.  The 64 bytes of
+// fp16 identity values of a chunk are copied by the thread itself with cp.async into its own slot of a small ring in
+// shared memory, ID_AHEAD chunks before they are needed (across tile boundaries), so the loads are in flight while
+// the MMAs run and while earlier chunks are computed; no other thread reads the slot, so cp.async.wait_group is the
+// only synchronisation.  Rows are ID_ROW_BYTES apart (64 + 16: conflict-free 16-byte reads across a warp).
+// (A variant that turns each 32 x 32 block through shared memory so that a lane owns a channel - parameters in
+// registers, contiguous 64-byte requests, warp votes for the sign words - was measured at 0.55x the speed of this
+// one: its 2-byte accesses and 32 votes per block cost more than the strided 16-byte accesses here.)
+constexpr int ID_AHEAD = 2;
+constexpr int ID_SLOTS = ID_AHEAD + 1;
+constexpr int ID_ROW_BYTES = 80;
+constexpr int ID_RING_BYTES = ID_SLOTS * BM * ID_ROW_BYTES;      // 30720
+
+// Queue the copy of one chunk (always commits a group, empty when there is nothing to copy).
+__device__ __forceinline__ void module_prefetch(const ConvProblem &p, uint32_t slot_addr, long row, int n0, bool live)
+{
+    if (p.identity && live) {
+        const uint16_t *src = p.identity + row * p.C_out + n0;
+#pragma unroll
+        for (int g = 0; g < 4; ++g) cp_async16(slot_addr + 16u * g, src + 8 * g, true);
+    }
+    cp_async_commit();
+}
+
+// One chunk: 32 consecutive output channels n0 .. n0+31 of one output row.
 //   t = dot * scale + shift;  u = t + identity;  r = u >= 0 ? u : slope * u;  y = fp16(r);  bit = (y + next_bias >= 0)
 // one fp32 operation per step, each rounded to nearest (no fused multiply-add), the sign taken of the stored
-// fp16 value.  Stores the 32 fp16 values (when `live`) and returns the 32 sign bits (bit i = channel n0 + i).
-// The channel count is a multiple of 32, so every 8-channel group is 16-byte aligned.
-__device__ __forceinline__ uint32_t module_chunk(const ConvProblem &p, const int (&dot)[32], long row, int n0, bool live)
+// fp16 value.  Reads the identity values from the thread's staging slot, stores the 32 fp16 values (when `live`)
+// and returns the 32 sign bits (bit i = channel n0 + i).  The channel count is a multiple of 32, so every
+// 8-channel group is 16-byte aligned.
+__device__ __forceinline__ uint32_t module_chunk(const ConvProblem &p, const int (&dot)[32], uint32_t slot_addr,
+                                                 long row, int n0, bool live)
 {
     uint32_t bits = 0;
     const long base = row * p.C_out + n0;
 #pragma unroll
     for (int g = 0; g < 4; ++g) {                           // 8 channels per group
         uint4 idv = make_uint4(0u, 0u, 0u, 0u);
-        if (p.identity && live) idv = __ldg(reinterpret_cast<const uint4 *>(p.identity + base + 8 * g));
+        if (p.identity && live) idv = ld_shared_v4(slot_addr + 16u * g);
         const uint32_t idw[4] = {idv.x, idv.y, idv.z, idv.w};
         uint32_t ow[4];
 #pragma unroll
