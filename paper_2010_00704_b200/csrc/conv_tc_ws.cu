@@ -425,6 +425,7 @@ conv_tc_ws_kernel(const ConvProblem p)
             constexpr uint32_t TAB_STAGE = (4 / GW) * 8u;
             constexpr uint32_t TSLOT_BYTES = SLOT_BYTES * KT;     // one staged tile: [KT][PROD_THREADS][16 B]
             const uint32_t tend = bits0 + PF * TSLOT_BYTES;
+            const int nk_last = p.kwords - 4 * (KT - 1);          // K words of the row's last stage (1..4)
             const TileStep gstep = make_tile_step(p, (uint32_t)BM * gridDim.x * G);
             RowCursor rc;
             rc.m = ((uint32_t)blockIdx.x + (uint32_t)grp * gridDim.x) * BM + (uint32_t)row;
@@ -435,7 +436,8 @@ conv_tc_ws_kernel(const ConvProblem p)
             auto issue = [&]() {
 #pragma unroll
                 for (int kt = 0; kt < KT; ++kt)
-                    gather_stage<GW>(p.x, rc, ktab_addr + (uint32_t)kt * TAB_STAGE, l_dst + (uint32_t)kt * SLOT_BYTES);
+                    gather_stage<GW>(p.x, rc, ktab_addr + (uint32_t)kt * TAB_STAGE, l_dst + (uint32_t)kt * SLOT_BYTES,
+                                     kt < KT - 1 ? 4 : (nk_last + GW - 1) / GW);
                 l_dst += TSLOT_BYTES;
                 if (l_dst == tend) l_dst = bits0;
                 --l_left;
@@ -463,11 +465,7 @@ conv_tc_ws_kernel(const ConvProblem p)
                     if (alive && !mbar_wait_warp(empty_bar(s), phase, abort_flag, p.err, ERR_PRODUCER_TIMEOUT)) alive = false;
                     if (alive) {
                         tc_fence_after();
-                        uint32_t v[32];
-                        const uint32_t wds[4] = {bits.x, bits.y, bits.z, bits.w};
-#pragma unroll
-                        for (int e = 0; e < 4; ++e) expand_a(wds[e], &v[8 * e]);
-                        tc_st32(st_addr0 + (uint32_t)s * 32u, v);
+                        expand_store_stage(st_addr0 + (uint32_t)s * 32u, bits, kt < KT - 1 ? 4 : nk_last);
                         tc_fence_before();
                         __syncwarp();
                         mbar_arrive_pred(full_bar(s), lane0);

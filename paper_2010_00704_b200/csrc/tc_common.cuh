@@ -280,6 +280,28 @@ __device__ __forceinline__ void expand_store_w_signed(uint32_t w, bool live, uin
     st_shared_v4(row_addr + (uint32_t)(((c + 1) ^ xr) << 4), o[4], o[5], o[6], o[7]);
 }
 
+// Expand the first nk (1..4) K words of a 128-bit stage into this lane's tensor-memory row (8 columns per word)
+// and wait for the stores.  A partial stage stores only its words: the MMAs skip the rest.
+__device__ __forceinline__ void expand_store_stage(uint32_t taddr, const uint4 &bits, int nk)
+{
+    const uint32_t wds[4] = {bits.x, bits.y, bits.z, bits.w};
+    if (nk >= 4) {
+        uint32_t v[32];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) expand_a(wds[e], &v[8 * e]);
+        tc_st32_nowait(taddr, v);
+    } else {
+#pragma unroll
+        for (int e = 0; e < 3; ++e)
+            if (e < nk) {                                   // warp-uniform
+                uint32_t v[8];
+                expand_a(wds[e], v);
+                tc_st8_nowait(taddr + 8u * e, v);
+            }
+    }
+    tc_wait_st();
+}
+
 // ---- implicit-im2col gather -----------------------------------------------------------------------
 // K is cut into units of GW words that never straddle a tap: GW = 4 (one 16-byte copy) when a pixel
 // is a multiple of four words, 2 when it is even, else 1.  The unit table holds, per unit, the word
@@ -370,9 +392,11 @@ __device__ __forceinline__ void cp_async_zfill(uint32_t dst, const void *src, ui
     else
         asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;" ::"r"(dst), "l"(src), "r"(nbytes) : "memory");
 }
-// One 128-bit stage (4 / GW units, table entries at `tab`) of the row `rc` -> 16 bytes at `dst`.
+// One 128-bit stage (4 / GW units, table entries at `tab`) of the row `rc` -> 16 bytes at `dst`.  Only the
+// first `nunits` units are copied (warp-uniform; the zero tail of K beyond the last word needs no copy when
+// nobody reads it).
 template <int GW>
-__device__ __forceinline__ void gather_stage(const uint32_t *x, const RowCursor &rc, uint32_t tab, uint32_t dst)
+__device__ __forceinline__ void gather_stage(const uint32_t *x, const RowCursor &rc, uint32_t tab, uint32_t dst, int nunits = 4)
 {
     constexpr int U = 4 / GW;
     uint32_t ent[2 * U];
@@ -386,6 +410,7 @@ __device__ __forceinline__ void gather_stage(const uint32_t *x, const RowCursor 
     }
 #pragma unroll
     for (int u = 0; u < U; ++u) {
+        if (u >= nunits) break;
         const bool ok = (rc.mask & ent[2 * u + 1]) != 0u;
         const int idx = ok ? rc.base + (int)ent[2 * u] : 0;
         cp_async_zfill<GW * 4>(dst + (uint32_t)(u * GW * 4), x + idx, ok ? (uint32_t)(GW * 4) : 0u);
