@@ -76,13 +76,17 @@ int make_conv_problem(ConvProblem &p, const void *x, const void *w, const int32_
 // Measured on B200 (bench.py --mode sweep):
 //   * C_out >= 256, or weights too large to keep expanded in shared memory: streaming tcgen05 engine;
 //   * 1x1 layer with C_in = 32 and C_out <= 32 (one XOR + popcount per output): CUDA-core pointwise kernel;
-//   * C_out <= 128 with K >= 64: weight-stationary tcgen05 engine;
+//   * C_out <= 128 with K >= 64, and wider layers with K <= 1152 and M >= 32768 (in 128-channel slices):
+//     weight-stationary tcgen05 engine;
 //   * other K = 32 layers: register-fed warp-level int8 engine;
 //   * the single-bit mma.sync and CUDA-core engines never win and serve as fallbacks.
 int auto_engine(const ConvProblem &p)
 {
     if (conv_lop3_pointwise_k32(p)) return BCNN_ENGINE_LOP3;
     if (p.C_out <= 128 && p.K >= 64 && conv_tc_ws_supports(p)) return BCNN_ENGINE_TC_WS;
+    // wider layers in slices of 128 output channels: ahead of the streaming engine while K is short and there are
+    // enough rows to share one slice's weights among many CTAs (K = 2304 ties, K = 512 at M = 12544 loses)
+    if (p.C_out > 128 && p.K <= 1152 && p.M >= 32768 && conv_tc_ws_supports(p)) return BCNN_ENGINE_TC_WS;
     if (p.C_out <= 64 && conv_mma_s8_supports(p)) return BCNN_ENGINE_MMA_S8;
     if (conv_tc_i8_supports(p)) return BCNN_ENGINE_TC_I8;
     if (conv_mma_b1_supports(p)) return BCNN_ENGINE_MMA_B1;

@@ -1,5 +1,6 @@
-// Weight-stationary variant of the tcgen05 engine for layers with few output channels and a
-// short K (C_out <= 128 and the expanded weights fit in shared memory).
+// Weight-stationary variant of the tcgen05 engine for layers with a short K: the expanded weights of up to
+// 128 output channels fit in shared memory.  Wider layers run as slices of 128 (or 64) output channels: a CTA
+// keeps one slice's weights, so the activations are expanded once per slice.
 //
 // Arithmetic.  Sign bits are expanded to bytes on chip; byte 4j+i of a 32-bit group carries bit j+8i.
 //   activations (unsigned bytes): 0 where the bit is clear, else 2^j (j <= 6) or 64 (j = 7)
@@ -112,7 +113,14 @@ conv_tc_ws_kernel(const ConvProblem p)
     const int ktiles = L.ktiles;
     constexpr int STAGES = C::STAGES;
     const int m_tiles = (p.M + BM - 1) / BM;
-    const int my_tiles = ((int)blockIdx.x < m_tiles) ? (m_tiles - 1 - (int)blockIdx.x) / (int)gridDim.x + 1 : 0;
+    // N slices: a CTA keeps the weights of one slice of BN output channels and walks row tiles mb, mb + mstride, ...
+    // (the grid is a multiple of the slice count)
+    const int n_tiles = (p.C_out + BN - 1) / BN;
+    const int n0 = ((int)blockIdx.x % n_tiles) * BN;
+    const int cn = min(BN, p.C_out - n0);                     // channels of this slice
+    const int mb = (int)blockIdx.x / n_tiles;
+    const int mstride = (int)gridDim.x / n_tiles;
+    const int my_tiles = (mb < m_tiles) ? (m_tiles - 1 - mb) / mstride + 1 : 0;
     const int total_items = my_tiles * ktiles;
 
     // shared-memory map (all 1024-byte aligned where the MMA reads)
@@ -152,20 +160,20 @@ conv_tc_ws_kernel(const ConvProblem p)
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
             const int kword = kt * 4 + e;
-            const bool live = kword < p.kwords && row < p.C_out;         // rows / K words beyond the problem: zero bytes
-            const uint32_t w = live ? __ldg(p.w + (long)row * p.kwords + kword) : 0u;
+            const bool live = kword < p.kwords && row < cn;              // rows / K words beyond the problem: zero bytes
+            const uint32_t w = live ? __ldg(p.w + (long)(n0 + row) * p.kwords + kword) : 0u;
             expand_store_w_signed(w, live, row_addr, row & 7, 2 * e);
         }
     }
     for (int c = tid; c < BN; c += C::THREADS) {
         int pop = 0;
-        if (c < p.C_out)
-            for (int kw = 0; kw < p.kwords; ++kw) pop += __popc(__ldg(p.w + (long)c * p.kwords + kw));
+        if (c < cn)
+            for (int kw = 0; kw < p.kwords; ++kw) pop += __popc(__ldg(p.w + (long)(n0 + c) * p.kwords + kw));
         // with acc = 64 * S:   int32: (acc >> 5) + (K - 2*pop)      fused: acc + 32*(K - 2*pop - thr) >= 0
         // (a threshold beyond +-(K + 1) decides like that bound; clamping keeps the constant inside int32)
         int cst = p.K - 2 * pop;
         if (FUSED) {
-            int t = c < p.C_out ? __ldg(p.thr + c) : 0;
+            int t = c < cn ? __ldg(p.thr + n0 + c) : 0;
             t = max(min(t, p.K + 1), -p.K - 1);
             cst = 32 * (cst - t);
         }
@@ -247,13 +255,13 @@ conv_tc_ws_kernel(const ConvProblem p)
         uint32_t buf_phase = 0;
         // module epilogue: chunk q of this thread's row sequence = (tile q / nch, chunk q % nch); its identity values
         // are staged ID_AHEAD chunks ahead in ring slot q % ID_SLOTS
-        const int nch = (p.C_out + 31) >> 5;
+        const int nch = (cn + 31) >> 5;
         const uint32_t id_row = idring + (uint32_t)erow * ID_ROW_BYTES;
         int pf_ti = 0, pf_ch = 0, pf_slot = 0, cur_slot = 0;
         auto prefetch_next = [&]() {
             if (pf_ti < my_tiles) {
-                const long row = (long)((int)blockIdx.x + pf_ti * (int)gridDim.x) * BM + erow;
-                module_prefetch(p, id_row + (uint32_t)pf_slot * (BM * ID_ROW_BYTES), row, pf_ch * 32, row < p.M);
+                const long row = (long)(mb + pf_ti * mstride) * BM + erow;
+                module_prefetch(p, id_row + (uint32_t)pf_slot * (BM * ID_ROW_BYTES), row, n0 + pf_ch * 32, row < p.M);
                 if (++pf_ch == nch) { pf_ch = 0; ++pf_ti; }
             } else {
                 cp_async_commit();
@@ -263,7 +271,7 @@ conv_tc_ws_kernel(const ConvProblem p)
         if (MODULE)
             for (int a = 0; a < ID_AHEAD; ++a) prefetch_next();
         for (int ti = 0; ti < my_tiles; ++ti) {
-            const int m_tile = (int)blockIdx.x + ti * (int)gridDim.x;
+            const int m_tile = mb + ti * mstride;
             const int em = m_tile * BM + erow;
             if (alive) alive = mbar_wait(tfull_bar(buf), buf_phase, abort_flag, p.err, ERR_EPILOGUE_TIMEOUT);
             alive = __all_sync(0xffffffffu, alive && !*abort_flag);
@@ -275,7 +283,7 @@ conv_tc_ws_kernel(const ConvProblem p)
             for (int ch = 0; ch < BN / 32; ++ch) {
                 const int col0 = ch * 32;
                 words[ch] = 0;
-                if (col0 < p.C_out) {                                 // warp-uniform
+                if (col0 < cn) {                                      // warp-uniform
                     uint32_t v[32];
                     tc_ld32(t_addr + (uint32_t)col0, v);
                     if (FUSED) {
@@ -301,11 +309,11 @@ conv_tc_ws_kernel(const ConvProblem p)
                         }
                         prefetch_next();
                         cp_async_wait<ID_AHEAD>();                    // this chunk's copy has landed
-                        words[ch] = module_chunk(p, dot, id_row + (uint32_t)cur_slot * (BM * ID_ROW_BYTES), em, col0, em < p.M);
+                        words[ch] = module_chunk(p, dot, id_row + (uint32_t)cur_slot * (BM * ID_ROW_BYTES), em, n0 + col0, em < p.M);
                         if (++cur_slot == ID_SLOTS) cur_slot = 0;
                     } else if (em < p.M) {
-                        int32_t *dst = static_cast<int32_t *>(p.out) + (long)em * p.C_out + col0;
-                        const bool vec = (p.C_out & 3) == 0 && (col0 + 32 <= p.C_out);
+                        int32_t *dst = static_cast<int32_t *>(p.out) + (long)em * p.C_out + n0 + col0;
+                        const bool vec = (p.C_out & 3) == 0 && (n0 + col0 + 32 <= p.C_out);
 #pragma unroll
                         for (int i4 = 0; i4 < 8; ++i4) {
                             const uint4 cc = ld_shared_v4(colc_addr + 4u * (col0 + 4 * i4));
@@ -317,7 +325,7 @@ conv_tc_ws_kernel(const ConvProblem p)
                             if (vec) {
                                 *reinterpret_cast<int4 *>(dst + 4 * i4) = o;
                             } else {
-                                const int n = col0 + 4 * i4;
+                                const int n = n0 + col0 + 4 * i4;
                                 if (n < p.C_out) dst[4 * i4] = o.x;
                                 if (n + 1 < p.C_out) dst[4 * i4 + 1] = o.y;
                                 if (n + 2 < p.C_out) dst[4 * i4 + 2] = o.z;
@@ -332,16 +340,16 @@ conv_tc_ws_kernel(const ConvProblem p)
             if (lane == 0) mbar_arrive(tempty_bar(buf));
             if (++buf == NBUF) { buf = 0; buf_phase ^= 1u; }
             if ((FUSED || (MODULE && p.out != nullptr)) && em < p.M) {
-                const int owords = p.C_out >> 5;
-                uint32_t *dst = static_cast<uint32_t *>(p.out) + (long)em * owords;
-                if (BN == 128 && owords == 4) {
+                const int owords = p.C_out >> 5, swords = cn >> 5;      // words of a row, of this slice
+                uint32_t *dst = static_cast<uint32_t *>(p.out) + (long)em * owords + (n0 >> 5);
+                if (BN == 128 && swords == 4 && (owords & 3) == 0) {
                     *reinterpret_cast<uint4 *>(dst) = make_uint4(words[0], words[1], words[2], words[3]);
-                } else if (BN >= 64 && owords == 2) {
+                } else if (BN >= 64 && swords == 2 && (owords & 1) == 0) {
                     *reinterpret_cast<uint2 *>(dst) = make_uint2(words[0], words[1]);
                 } else {
 #pragma unroll
                     for (int ch = 0; ch < BN / 32; ++ch)
-                        if (ch < owords) dst[ch] = words[ch];
+                        if (ch < swords) dst[ch] = words[ch];
                 }
             }
         }
@@ -359,14 +367,14 @@ conv_tc_ws_kernel(const ConvProblem p)
         const uint32_t bits0 = bits_ring + (uint32_t)ptid * 16u, bits_end = bits0 + PF * SLOT_BYTES;
         const uint32_t st_addr0 = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)C::A_COL0;
         const uint32_t lane0 = lane == 0 ? 1u : 0u;
-        const TileStep step = make_tile_step(p, (uint32_t)BM * gridDim.x);
+        const TileStep step = make_tile_step(p, (uint32_t)(BM * mstride));
 
         auto produce = [&](auto gw_tag) {
             constexpr int GW = decltype(gw_tag)::value;
             constexpr uint32_t TAB_STAGE = (4 / GW) * 8u;        // table bytes per stage
             // ---- load cursor
             RowCursor rc;
-            rc.m = (uint32_t)blockIdx.x * BM + (uint32_t)row;
+            rc.m = (uint32_t)mb * BM + (uint32_t)row;
             row_locate(p, rc);
             int l_kt = grp;
             int l_left = total_items > grp ? (total_items - grp + G - 1) / G : 0;
@@ -426,9 +434,9 @@ conv_tc_ws_kernel(const ConvProblem p)
             constexpr uint32_t TSLOT_BYTES = SLOT_BYTES * KT;     // one staged tile: [KT][PROD_THREADS][16 B]
             const uint32_t tend = bits0 + PF * TSLOT_BYTES;
             const int nk_last = p.kwords - 4 * (KT - 1);          // K words of the row's last stage (1..4)
-            const TileStep gstep = make_tile_step(p, (uint32_t)BM * gridDim.x * G);
+            const TileStep gstep = make_tile_step(p, (uint32_t)(BM * mstride * G));
             RowCursor rc;
-            rc.m = ((uint32_t)blockIdx.x + (uint32_t)grp * gridDim.x) * BM + (uint32_t)row;
+            rc.m = (uint32_t)(mb + grp * mstride) * BM + (uint32_t)row;
             row_locate(p, rc);
             row_window(p, gstep, rc);
             int l_left = my_tiles > grp ? (my_tiles - grp + G - 1) / G : 0;
@@ -513,7 +521,11 @@ int launch_ws(const ConvProblem &p0, cudaStream_t stream)
     const WsLayout L = ws_layout<BN, G, DUAL>(p.kwords, p.mode == 2);
     const long m_tiles = ((long)p.M + BM - 1) / BM;
     const long slots = (long)sms * C::CTAS_PER_SM;
-    const unsigned grid = (unsigned)(m_tiles < slots ? m_tiles : slots);
+    const long n_tiles = (p.C_out + BN - 1) / BN;
+    long per_slice = slots / n_tiles;                         // CTAs that share one slice of the weights
+    if (per_slice < 1) return BCNN_ERR_UNSUPPORTED;
+    if (per_slice > m_tiles) per_slice = m_tiles;
+    const unsigned grid = (unsigned)(per_slice * n_tiles);
     void (*k)(const ConvProblem) = p.mode == 2 ? conv_tc_ws_kernel<BN, G, DUAL, 2> : (p.mode == 1 ? conv_tc_ws_kernel<BN, G, DUAL, 1> : conv_tc_ws_kernel<BN, G, DUAL, 0>);
     // the attribute is a property of the kernel, not of the launch: always the configuration's limit, so
     // that a captured launch stays valid whatever later calls with other shapes ask for
@@ -535,12 +547,14 @@ bool fits(const ConvProblem &p)
 bool conv_tc_ws_supports(const ConvProblem &p)
 {
     if (p.mode != 0 && (p.C_out % 32 != 0)) return false;
-    if (p.C_out > 128 || p.kh * p.kw > 31 || p.K > (1 << 16)) return false;
+    if (p.kh * p.kw > 31 || p.K > (1 << 16)) return false;
     // rows address the input by 32-bit word offsets
     if ((long)p.B * p.H * p.W * p.cw >= (1L << 31)) return false;
     if (p.C_out <= 32) return fits<32, 4, false>(p);
     if (p.C_out <= 64) return fits<64, 4, false>(p);
-    return fits<128, 4, false>(p) || fits<128, 2, false>(p);
+    if (fits<128, 4, false>(p) || fits<128, 2, false>(p)) return p.C_out <= 128 * 64;
+    // wider layers whose 128-channel slice of the weights does not fit: 64-channel slices
+    return p.C_out > 128 && p.C_out <= 64 * 64 && fits<64, 4, false>(p);
 }
 
 int launch_conv_tc_ws(const ConvProblem &p, cudaStream_t stream)
@@ -550,9 +564,11 @@ int launch_conv_tc_ws(const ConvProblem &p, cudaStream_t stream)
     // per SM (two issuers) when the resident weights leave room for it
     if (p.C_out <= 32) return fits<32, 2, true>(p) ? launch_ws<32, 2, true>(p, stream) : launch_ws<32, 4, false>(p, stream);
     if (p.C_out <= 64) return fits<64, 2, true>(p) ? launch_ws<64, 2, true>(p, stream) : launch_ws<64, 4, false>(p, stream);
+    // C_out > 128: slices of 128 (or 64) output channels, each CTA keeps one slice's weights
     if (fits<128, 2, true>(p)) return launch_ws<128, 2, true>(p, stream);
     if (fits<128, 4, false>(p)) return launch_ws<128, 4, false>(p, stream);
-    return launch_ws<128, 2, false>(p, stream);     // long K: fewer producer groups, smaller staging ring
+    if (fits<128, 2, false>(p)) return launch_ws<128, 2, false>(p, stream);     // long K: fewer producer groups, smaller staging ring
+    return fits<64, 2, true>(p) ? launch_ws<64, 2, true>(p, stream) : launch_ws<64, 4, false>(p, stream);
 }
 
 }  // namespace bcnn
