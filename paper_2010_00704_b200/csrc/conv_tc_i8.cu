@@ -517,7 +517,18 @@ int launch_conv_tc_i8(const ConvProblem &p, cudaStream_t stream)
     // 256-wide tiles have a single accumulator buffer (tensor memory also holds the activation
     // ring), so their epilogue is not overlapped: worth it only when the K loop is long
     // (the module epilogue's staging ring only fits beside the 128-wide tiles' weight ring)
-    if (p.C_out > 128 && p.kwords >= 24 && p.mode != 2) return launch_bn<256>(p, stream);
+    if (p.C_out > 128 && p.kwords >= 24 && p.mode != 2) {
+        // ... unless the narrower tiles fill the last wave so much better that they win anyway: a 128-wide tile
+        // costs about 0.6 of a 256-wide one (measured on the K = 2304 and K = 4608 layers)
+        int dev = 0, sms = 148;
+        cudaGetDevice(&dev);
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+        const long m_tiles = ((long)p.M + BM - 1) / BM;
+        const long waves256 = (m_tiles * ((p.C_out + 255) / 256) + sms - 1) / sms;
+        const long waves128 = (m_tiles * ((p.C_out + 127) / 128) + sms - 1) / sms;
+        if (10 * waves256 <= 6 * waves128) return launch_bn<256>(p, stream);
+        return launch_bn<128>(p, stream);
+    }
     return launch_bn<128>(p, stream);
 }
 
