@@ -553,7 +553,7 @@ def run_paper1x1(args):
     for l, count in convs:
         ms = float(np.mean([a.elapsed_time(b) for a, b in per[l.name]]))
         shapes.append({"layer": l.name, "count": count, "M": l.M(B), "N": l.C_out, "K": l.K,
-                       "engine": ("tc_ws" if l.K >= 64 and l.C_out <= 128 else "tc_i8") if module
+                       "engine": "tc_ws" if module
                        else binding.bcnn_auto_engine(B, l.H, l.W, l.C_in, l.C_out, 1, 1, 1, 0),
                        "ms_per_launch": ms, "tops": l.ops(B) / (ms / 1e3) / 1e12})
         # algorithmic bytes: packed input + packed output (+ fp16 identity read and fp16 map written by the module)

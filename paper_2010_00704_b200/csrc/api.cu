@@ -207,8 +207,9 @@ int bcnn_conv2d_b1_module(const void *x_bits, const void *w_bits, const float *b
     p.identity = static_cast<const uint16_t *>(identity);
     p.y_real = static_cast<uint16_t *>(y_real);
     p.out = y_bits;
-    // the two tcgen05 engines carry this epilogue
-    if (p.C_out <= 128 && p.K >= 64 && conv_tc_ws_supports(p)) return launch_conv_tc_ws(p, static_cast<cudaStream_t>(stream));
+    // the two tcgen05 engines carry this epilogue; it is bound by the epilogue warps, of which the weight-stationary
+    // engine has twice as many per SM whenever two of its CTAs fit (wider layers run as 128-channel slices)
+    if (conv_tc_ws_supports(p)) return launch_conv_tc_ws(p, static_cast<cudaStream_t>(stream));
     return launch_conv_tc_i8(p, static_cast<cudaStream_t>(stream));
 }
 
