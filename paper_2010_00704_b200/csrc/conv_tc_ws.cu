@@ -33,8 +33,7 @@ namespace {
 
 using namespace tc;
 
-constexpr int EPI_WARPS = 4;
-constexpr int FIRST_PRODUCER_THREAD = 32 * (1 + EPI_WARPS);
+constexpr int EPI_WARPS = 4;              // warps of one epilogue team (one per tensor-memory lane quadrant)
 constexpr int PF = 3;                     // packed-word stages in flight per producer thread
 constexpr int MAX_SMEM = 227 * 1024;
 
@@ -43,7 +42,11 @@ constexpr int ERR_MMA_TIMEOUT = 112;
 constexpr int ERR_EPILOGUE_TIMEOUT = 113;
 
 // DUAL: two CTAs share an SM (two independent MMA issuers), each with half of tensor memory.
-template <int BN, int G, bool DUAL> struct Cfg {
+// TEAMS: epilogue teams of four warps; team t takes the tiles t, t + TEAMS, ... of the CTA (their accumulator
+// buffers are then a fixed subset, so NBUF is a multiple of TEAMS).  Two teams serve the module epilogue, which is
+// bound by the epilogue warps.
+template <int BN, int G, bool DUAL, int TEAMS = 1> struct Cfg {
+    static constexpr int FIRST_PRODUCER_THREAD = 32 * (1 + EPI_WARPS * TEAMS);
     static constexpr int BNX = BN;
     static constexpr int PROD_THREADS = G * BM;
     // Tensor memory (512 columns): NBUF accumulator buffers of BNX columns, then the activation ring,
@@ -70,10 +73,10 @@ struct WsLayout {
     int smem;         // dynamic shared memory in bytes
 };
 
-template <int BN, int G, bool DUAL>
+template <int BN, int G, bool DUAL, int TEAMS = 1>
 __host__ __device__ inline WsLayout ws_layout(int kwords, bool module)
 {
-    using C = Cfg<BN, G, DUAL>;
+    using C = Cfg<BN, G, DUAL, TEAMS>;
     WsLayout l;
     l.ktiles = (kwords + 3) >> 2;
     // Short K: a producer group takes whole tiles in turn instead of single stages, so the per-tile work
@@ -83,7 +86,7 @@ __host__ __device__ inline WsLayout ws_layout(int kwords, bool module)
     l.row_kt = (l.ktiles <= 3 && C::STAGES >= (G - 1) * l.ktiles + 1) ? l.ktiles : 0;
     l.bits_bytes = C::BITS_BYTES * (l.row_kt ? l.row_kt : 1);
     l.smem = 1024 + l.ktiles * C::W_TILE_BYTES + l.bits_bytes + BN * 4 + l.ktiles * 32;
-    if (module) l.smem += ID_RING_BYTES + 16;                 // identity staging ring of the module epilogue
+    if (module) l.smem += TEAMS * ID_RING_BYTES + 16;         // identity staging rings of the module epilogue
     // Tensor memory is shared out by the resident CTAs (all 512 columns, or 256 each for two): ask
     // for enough shared memory that no further CTA of this kernel fits on the SM (it would sit in
     // tcgen05.alloc until a neighbour exits).
@@ -92,11 +95,12 @@ __host__ __device__ inline WsLayout ws_layout(int kwords, bool module)
     return l;
 }
 
-template <int BN, int G, bool DUAL, int MODE>
-__global__ void __launch_bounds__(Cfg<BN, G, DUAL>::BOUND_THREADS, Cfg<BN, G, DUAL>::CTAS_PER_SM)
+template <int BN, int G, bool DUAL, int MODE, int TEAMS = 1>
+__global__ void __launch_bounds__(Cfg<BN, G, DUAL, TEAMS>::BOUND_THREADS, Cfg<BN, G, DUAL, TEAMS>::CTAS_PER_SM)
 conv_tc_ws_kernel(const ConvProblem p)
 {
-    using C = Cfg<BN, G, DUAL>;
+    using C = Cfg<BN, G, DUAL, TEAMS>;
+    static_assert(C::NBUF % TEAMS == 0, "a team's tiles must map to a fixed set of accumulator buffers");
     constexpr bool FUSED = MODE == 1, MODULE = MODE == 2;
     constexpr int BNX = C::BNX;
     constexpr int NBUF = C::NBUF;
@@ -109,7 +113,7 @@ conv_tc_ws_kernel(const ConvProblem p)
 
     const int tid = threadIdx.x;
     const int warp = tid >> 5, lane = tid & 31;
-    const WsLayout L = ws_layout<BN, G, DUAL>(p.kwords, MODULE);
+    const WsLayout L = ws_layout<BN, G, DUAL, TEAMS>(p.kwords, MODULE);
     const int ktiles = L.ktiles;
     constexpr int STAGES = C::STAGES;
     const int m_tiles = (p.M + BM - 1) / BM;
@@ -246,23 +250,22 @@ conv_tc_ws_kernel(const ConvProblem p)
             }
             if (++buf == NBUF) { buf = 0; buf_phase ^= 1u; }
         }
-    } else if (warp <= EPI_WARPS) {
+    } else if (warp <= EPI_WARPS * TEAMS) {
         // ------------------------------------------------------------------ epilogue
         const int quad = warp & 3;
         const int erow = quad * 32 + lane;
+        const int team = (warp - 1) >> 2;                        // takes the tiles team, team + TEAMS, ...
         bool alive = true;
-        int buf = 0;
-        uint32_t buf_phase = 0;
         // module epilogue: chunk q of this thread's row sequence = (tile q / nch, chunk q % nch); its identity values
         // are staged ID_AHEAD chunks ahead in ring slot q % ID_SLOTS
         const int nch = (cn + 31) >> 5;
-        const uint32_t id_row = idring + (uint32_t)erow * ID_ROW_BYTES;
-        int pf_ti = 0, pf_ch = 0, pf_slot = 0, cur_slot = 0;
+        const uint32_t id_row = idring + (uint32_t)team * ID_RING_BYTES + (uint32_t)erow * ID_ROW_BYTES;
+        int pf_ti = team, pf_ch = 0, pf_slot = 0, cur_slot = 0;
         auto prefetch_next = [&]() {
             if (pf_ti < my_tiles) {
                 const long row = (long)(mb + pf_ti * mstride) * BM + erow;
                 module_prefetch(p, id_row + (uint32_t)pf_slot * (BM * ID_ROW_BYTES), row, n0 + pf_ch * 32, row < p.M);
-                if (++pf_ch == nch) { pf_ch = 0; ++pf_ti; }
+                if (++pf_ch == nch) { pf_ch = 0; pf_ti += TEAMS; }
             } else {
                 cp_async_commit();
             }
@@ -270,7 +273,9 @@ conv_tc_ws_kernel(const ConvProblem p)
         };
         if (MODULE)
             for (int a = 0; a < ID_AHEAD; ++a) prefetch_next();
-        for (int ti = 0; ti < my_tiles; ++ti) {
+        for (int ti = team; ti < my_tiles; ti += TEAMS) {
+            const int buf = ti % NBUF;                            // tiles use the accumulator buffers in turn
+            const uint32_t buf_phase = (uint32_t)(ti / NBUF) & 1u;
             const int m_tile = mb + ti * mstride;
             const int em = m_tile * BM + erow;
             if (alive) alive = mbar_wait(tfull_bar(buf), buf_phase, abort_flag, p.err, ERR_EPILOGUE_TIMEOUT);
@@ -338,7 +343,6 @@ conv_tc_ws_kernel(const ConvProblem p)
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(tempty_bar(buf));
-            if (++buf == NBUF) { buf = 0; buf_phase ^= 1u; }
             if ((FUSED || (MODULE && p.out != nullptr)) && em < p.M) {
                 const int owords = p.C_out >> 5, swords = cn >> 5;      // words of a row, of this slice
                 uint32_t *dst = static_cast<uint32_t *>(p.out) + (long)em * owords + (n0 >> 5);
@@ -359,7 +363,7 @@ conv_tc_ws_kernel(const ConvProblem p)
         // Group g takes items g, g + G, ... of the CTA's flattened (tile, stage) list.  Per item a
         // thread copies its row's 128 bits of K into its staging slot (PF items ahead), then expands
         // the oldest staged item into the ring slot of tensor memory.
-        const int ptid = tid - FIRST_PRODUCER_THREAD;
+        const int ptid = tid - C::FIRST_PRODUCER_THREAD;
         const int grp = ptid >> 7;                               // group = 4 consecutive warps
         const int quad = warp & 3;                               // tensor-memory lane quadrant this warp may write
         const int row = quad * 32 + lane;                        // the four warps of a group cover rows 0..127
@@ -509,7 +513,7 @@ conv_tc_ws_kernel(const ConvProblem p)
     }
 }
 
-template <int BN, int G, bool DUAL>
+template <int BN, int G, bool DUAL, int TEAMS = 1>
 int launch_ws(const ConvProblem &p0, cudaStream_t stream)
 {
     ConvProblem p = p0;
@@ -517,8 +521,8 @@ int launch_ws(const ConvProblem &p0, cudaStream_t stream)
     int dev = 0, sms = 148;
     cudaGetDevice(&dev);
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-    using C = Cfg<BN, G, DUAL>;
-    const WsLayout L = ws_layout<BN, G, DUAL>(p.kwords, p.mode == 2);
+    using C = Cfg<BN, G, DUAL, TEAMS>;
+    const WsLayout L = ws_layout<BN, G, DUAL, TEAMS>(p.kwords, p.mode == 2);
     const long m_tiles = ((long)p.M + BM - 1) / BM;
     const long slots = (long)sms * C::CTAS_PER_SM;
     const long n_tiles = (p.C_out + BN - 1) / BN;
@@ -526,7 +530,8 @@ int launch_ws(const ConvProblem &p0, cudaStream_t stream)
     if (per_slice < 1) return BCNN_ERR_UNSUPPORTED;
     if (per_slice > m_tiles) per_slice = m_tiles;
     const unsigned grid = (unsigned)(per_slice * n_tiles);
-    void (*k)(const ConvProblem) = p.mode == 2 ? conv_tc_ws_kernel<BN, G, DUAL, 2> : (p.mode == 1 ? conv_tc_ws_kernel<BN, G, DUAL, 1> : conv_tc_ws_kernel<BN, G, DUAL, 0>);
+    void (*k)(const ConvProblem) = p.mode == 2 ? conv_tc_ws_kernel<BN, G, DUAL, 2, TEAMS>
+                                   : (p.mode == 1 ? conv_tc_ws_kernel<BN, G, DUAL, 1, TEAMS> : conv_tc_ws_kernel<BN, G, DUAL, 0, TEAMS>);
     // the attribute is a property of the kernel, not of the launch: always the configuration's limit, so
     // that a captured launch stays valid whatever later calls with other shapes ask for
     if (cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, DUAL ? 113 * 1024 : MAX_SMEM - 1024) != cudaSuccess) return BCNN_ERR_CUDA;
@@ -536,10 +541,10 @@ int launch_ws(const ConvProblem &p0, cudaStream_t stream)
 
 // The expanded weights, the packed-word staging ring and the tables must fit in shared memory
 // (in half of it when two CTAs share an SM).
-template <int BN, int G, bool DUAL>
+template <int BN, int G, bool DUAL, int TEAMS = 1>
 bool fits(const ConvProblem &p)
 {
-    return ws_layout<BN, G, DUAL>(p.kwords, p.mode == 2).smem <= (DUAL ? 113 * 1024 : MAX_SMEM - 1024);
+    return ws_layout<BN, G, DUAL, TEAMS>(p.kwords, p.mode == 2).smem <= (DUAL ? 113 * 1024 : MAX_SMEM - 1024);
 }
 
 }  // namespace
@@ -560,6 +565,12 @@ bool conv_tc_ws_supports(const ConvProblem &p)
 int launch_conv_tc_ws(const ConvProblem &p, cudaStream_t stream)
 {
     if (!conv_tc_ws_supports(p)) return BCNN_ERR_UNSUPPORTED;
+    // module epilogue: bound by the epilogue warps, so two teams of them, one producer group and two CTAs per SM;
+    // layers wider than 64 channels run as 64-channel slices (two accumulator buffers are needed for two teams)
+    if (p.mode == 2) {
+        if (p.C_out <= 32 && fits<32, 1, true, 2>(p)) return launch_ws<32, 1, true, 2>(p, stream);
+        if (p.C_out > 32 && fits<64, 1, true, 2>(p)) return launch_ws<64, 1, true, 2>(p, stream);
+    }
     // narrow layers: the per-stage cost of issuing MMAs exceeds their execution time, so two CTAs
     // per SM (two issuers) when the resident weights leave room for it
     if (p.C_out <= 32) return fits<32, 2, true>(p) ? launch_ws<32, 2, true>(p, stream) : launch_ws<32, 4, false>(p, stream);
