@@ -184,7 +184,7 @@ conv_tc_i8_kernel(const ConvProblem p, const int ktab_words)
         uint32_t buf_phase = 0;
         // module epilogue: the identity values of this thread's row are staged ID_AHEAD live chunks ahead (a chunk is
         // live when its first channel exists), in ring slot (live chunk number) % ID_SLOTS
-        const uint32_t id_row = idring + (uint32_t)erow * ID_ROW_BYTES;
+        const uint32_t id_warp = idring + (uint32_t)(quad * 32) * ID_ROW_BYTES;   // slot 0, the warp's first row
         int pf_ti = 0, pf_ch = 0, pf_slot = 0, cur_slot = 0;
         auto prefetch_next = [&]() {
             bool queued = false;
@@ -193,8 +193,7 @@ conv_tc_i8_kernel(const ConvProblem p, const int ktab_words)
                 const int nt = t / m_tiles, mt = t - nt * m_tiles;
                 const int n = nt * BN + pf_ch * 32;
                 if (n < p.C_out) {
-                    const long row = (long)mt * BM + erow;
-                    module_prefetch(p, id_row + (uint32_t)pf_slot * (BM * ID_ROW_BYTES), row, n, row < p.M);
+                    module_prefetch(p, id_warp + (uint32_t)pf_slot * (BM * ID_ROW_BYTES), (long)mt * BM + quad * 32, n, lane);
                     queued = true;
                 }
                 if (++pf_ch == BN / 32) { pf_ch = 0; ++pf_ti; }
@@ -266,7 +265,7 @@ conv_tc_i8_kernel(const ConvProblem p, const int ktab_words)
                         }
                         prefetch_next();
                         cp_async_wait<ID_AHEAD>();                    // this chunk's copy has landed
-                        words[ch] = module_chunk(p, dot, id_row + (uint32_t)cur_slot * (BM * ID_ROW_BYTES), em, n0 + col0, em < p.M);
+                        words[ch] = module_chunk(p, dot, id_warp + (uint32_t)cur_slot * (BM * ID_ROW_BYTES), (long)em - lane, n0 + col0, lane);
                         if (++cur_slot == ID_SLOTS) cur_slot = 0;
                     } else if (em < p.M) {
                         int32_t *dst = static_cast<int32_t *>(p.out) + (long)em * p.C_out + n0 + col0;

@@ -259,12 +259,12 @@ conv_tc_ws_kernel(const ConvProblem p)
         // module epilogue: chunk q of this thread's row sequence = (tile q / nch, chunk q % nch); its identity values
         // are staged ID_AHEAD chunks ahead in ring slot q % ID_SLOTS
         const int nch = (cn + 31) >> 5;
-        const uint32_t id_row = idring + (uint32_t)team * ID_RING_BYTES + (uint32_t)erow * ID_ROW_BYTES;
+        const uint32_t id_warp = idring + (uint32_t)team * ID_RING_BYTES + (uint32_t)(quad * 32) * ID_ROW_BYTES;   // slot 0, the warp's first row
         int pf_ti = team, pf_ch = 0, pf_slot = 0, cur_slot = 0;
         auto prefetch_next = [&]() {
             if (pf_ti < my_tiles) {
-                const long row = (long)(mb + pf_ti * mstride) * BM + erow;
-                module_prefetch(p, id_row + (uint32_t)pf_slot * (BM * ID_ROW_BYTES), row, n0 + pf_ch * 32, row < p.M);
+                const long row0 = (long)(mb + pf_ti * mstride) * BM + quad * 32;
+                module_prefetch(p, id_warp + (uint32_t)pf_slot * (BM * ID_ROW_BYTES), row0, n0 + pf_ch * 32, lane);
                 if (++pf_ch == nch) { pf_ch = 0; pf_ti += TEAMS; }
             } else {
                 cp_async_commit();
@@ -314,7 +314,7 @@ conv_tc_ws_kernel(const ConvProblem p)
                         }
                         prefetch_next();
                         cp_async_wait<ID_AHEAD>();                    // this chunk's copy has landed
-                        words[ch] = module_chunk(p, dot, id_row + (uint32_t)cur_slot * (BM * ID_ROW_BYTES), em, n0 + col0, em < p.M);
+                        words[ch] = module_chunk(p, dot, id_warp + (uint32_t)cur_slot * (BM * ID_ROW_BYTES), (long)em - lane, n0 + col0, lane);
                         if (++cur_slot == ID_SLOTS) cur_slot = 0;
                     } else if (em < p.M) {
                         int32_t *dst = static_cast<int32_t *>(p.out) + (long)em * p.C_out + n0 + col0;

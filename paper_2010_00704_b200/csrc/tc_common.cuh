@@ -420,10 +420,10 @@ __device__ __forceinline__ void gather_stage(const uint32_t *x, const RowCursor 
 // Convolution-module epilogue (Section 4.2.1).
 //
 // Identity staging: an epilogue thread owns one output row and walks its 32-channel chunks in order.  The 64 bytes of
-// fp16 identity values of a chunk are copied by the thread itself with cp.async into its own slot of a small ring in
-// shared memory, ID_AHEAD chunks before they are needed (across tile boundaries), so the loads are in flight while
-// the MMAs run and while earlier chunks are computed; no other thread reads the slot, so cp.async.wait_group is the
-// only synchronisation.  Rows are ID_ROW_BYTES apart (64 + 16: conflict-free 16-byte reads across a warp).
+// fp16 identity values of a chunk are copied with cp.async into the row's slot of a small ring in shared memory,
+// ID_AHEAD chunks before they are needed (across tile boundaries), so the loads are in flight while the MMAs run
+// and while earlier chunks are computed.  Rows are ID_ROW_BYTES apart (64 + 16: conflict-free 16-byte accesses
+// across a warp, both one row per lane and four lanes per row).
 // (A variant that turns each 32 x 32 block through shared memory so that a lane owns a channel - parameters in
 // registers, contiguous 64-byte requests, warp votes for the sign words - was measured at 0.55x the speed of this
 // one: its 2-byte accesses and 32 votes per block cost more than the strided 16-byte accesses here.)
@@ -432,32 +432,42 @@ constexpr int ID_SLOTS = ID_AHEAD + 1;
 constexpr int ID_ROW_BYTES = 80;
 constexpr int ID_RING_BYTES = ID_SLOTS * BM * ID_ROW_BYTES;      // 30720
 
-// Queue the copy of one chunk (always commits a group, empty when there is nothing to copy).
-__device__ __forceinline__ void module_prefetch(const ConvProblem &p, uint32_t slot_addr, long row, int n0, bool live)
+// Queue the copy of one chunk for the 32 rows of this warp (always commits a group, empty when there is nothing to
+// copy).  The warp copies cooperatively: lane l fetches 16-byte part l % 4 of rows l / 4 + 8 i, so that one
+// instruction touches 8 rows x 64 contiguous bytes instead of 32 rows x 16 bytes; `warp_slot` is the slot of the
+// warp's first row, `row0` that row.  After cp.async.wait_group a __syncwarp makes all lanes' copies visible.
+__device__ __forceinline__ void module_prefetch(const ConvProblem &p, uint32_t warp_slot, long row0, int n0, int lane)
 {
-    if (p.identity && live) {
-        const uint16_t *src = p.identity + row * p.C_out + n0;
+    if (p.identity) {
 #pragma unroll
-        for (int g = 0; g < 4; ++g) cp_async16(slot_addr + 16u * g, src + 8 * g, true);
+        for (int i = 0; i < 4; ++i) {
+            const int r = (lane >> 2) + 8 * i;
+            const long row = row0 + r;
+            const bool ok = row < p.M;
+            cp_async16(warp_slot + (uint32_t)(r * ID_ROW_BYTES + (lane & 3) * 16),
+                       p.identity + (ok ? row * p.C_out + n0 + 8 * (lane & 3) : 0), ok);
+        }
     }
     cp_async_commit();
 }
 
-// One chunk: 32 consecutive output channels n0 .. n0+31 of one output row.
+// One chunk: 32 consecutive output channels n0 .. n0+31 of the warp's 32 output rows, lane = row.
 //   t = dot * scale + shift;  u = t + identity;  r = u >= 0 ? u : slope * u;  y = fp16(r);  bit = (y + next_bias >= 0)
 // one fp32 operation per step, each rounded to nearest (no fused multiply-add), the sign taken of the stored
-// fp16 value.  Reads the identity values from the thread's staging slot, stores the 32 fp16 values (when `live`)
-// and returns the 32 sign bits (bit i = channel n0 + i).  The channel count is a multiple of 32, so every
-// 8-channel group is 16-byte aligned.
-__device__ __forceinline__ uint32_t module_chunk(const ConvProblem &p, const int (&dot)[32], uint32_t slot_addr,
-                                                 long row, int n0, bool live)
+// fp16 value.  Reads the identity values from the row's staging slot, writes the 32 fp16 values back into the
+// same slot, from where the warp stores them cooperatively (same 8 rows x 64 bytes per instruction), and returns
+// the 32 sign bits of the lane's row (bit i = channel n0 + i).  The channel count is a multiple of 32, so every
+// 8-channel group is 16-byte aligned.  All 32 lanes must call it.
+__device__ __forceinline__ uint32_t module_chunk(const ConvProblem &p, const int (&dot)[32], uint32_t warp_slot,
+                                                 long row0, int n0, int lane)
 {
     uint32_t bits = 0;
-    const long base = row * p.C_out + n0;
+    const uint32_t slot_addr = warp_slot + (uint32_t)(lane * ID_ROW_BYTES);
+    __syncwarp();                                           // the cooperative copies of all lanes have landed
 #pragma unroll
     for (int g = 0; g < 4; ++g) {                           // 8 channels per group
         uint4 idv = make_uint4(0u, 0u, 0u, 0u);
-        if (p.identity && live) idv = ld_shared_v4(slot_addr + 16u * g);
+        if (p.identity) idv = ld_shared_v4(slot_addr + 16u * g);
         const uint32_t idw[4] = {idv.x, idv.y, idv.z, idv.w};
         uint32_t ow[4];
 #pragma unroll
@@ -488,8 +498,17 @@ __device__ __forceinline__ uint32_t module_chunk(const ConvProblem &p, const int
             ow[2 * h] = (uint32_t)hv[0] | ((uint32_t)hv[1] << 16);
             ow[2 * h + 1] = (uint32_t)hv[2] | ((uint32_t)hv[3] << 16);
         }
-        if (live) *reinterpret_cast<uint4 *>(p.y_real + base + 8 * g) = make_uint4(ow[0], ow[1], ow[2], ow[3]);
+        st_shared_v4(slot_addr + 16u * g, ow[0], ow[1], ow[2], ow[3]);
     }
+    __syncwarp();                                           // the rows of all lanes are staged
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int r = (lane >> 2) + 8 * i;
+        const long row = row0 + r;
+        const uint4 v = ld_shared_v4(warp_slot + (uint32_t)(r * ID_ROW_BYTES + (lane & 3) * 16));
+        if (row < p.M) *reinterpret_cast<uint4 *>(p.y_real + row * p.C_out + n0 + 8 * (lane & 3)) = v;
+    }
+    __syncwarp();                                           // the slot may be refilled
     return bits;
 }
 
