@@ -570,6 +570,7 @@ int launch_conv_tc_ws(const ConvProblem &p, cudaStream_t stream)
     if (p.mode == 2) {
         if (p.C_out <= 32 && fits<32, 1, true, 2>(p)) return launch_ws<32, 1, true, 2>(p, stream);
         if (p.C_out > 32 && fits<64, 1, true, 2>(p)) return launch_ws<64, 1, true, 2>(p, stream);
+        if (p.C_out > 32 && p.C_out <= 32 * 64 && fits<32, 1, true, 2>(p)) return launch_ws<32, 1, true, 2>(p, stream);   // long K: 32-channel slices
     }
     // narrow layers: the per-stage cost of issuing MMAs exceeds their execution time, so two CTAs
     // per SM (two issuers) when the resident weights leave room for it
