@@ -57,11 +57,13 @@ template <int BN> struct Cfg {
 };
 
 template <int BN>
-__host__ __device__ inline int smem_bytes(int ktab_words, bool module = false)
+__host__ __device__ inline int smem_bytes(int ktab_words, int mode = 1)
 {
     using C = Cfg<BN>;
-    // module epilogue: + the identity staging ring
-    return 1024 + C::STAGES * C::W_BYTES + C::BITS_BYTES + C::CONST_BYTES + ktab_words * 4 + (module ? ID_RING_BYTES + 16 : 0);
+    // module epilogue: + the identity staging ring; int32 output of the 128-wide tiles: + the store staging tiles
+    // (both only used where they fit: 128-wide tiles)
+    return 1024 + C::STAGES * C::W_BYTES + C::BITS_BYTES + C::CONST_BYTES + ktab_words * 4 +
+           (mode == 2 ? ID_RING_BYTES + 16 : 0) + (mode == 0 && BN == 128 ? EPI_WARPS * I32_TILE_BYTES + 16 : 0);
 }
 
 template <int BN, int MODE>
@@ -185,6 +187,8 @@ conv_tc_i8_kernel(const ConvProblem p, const int ktab_words)
         // module epilogue: the identity values of this thread's row are staged ID_AHEAD live chunks ahead (a chunk is
         // live when its first channel exists), in ring slot (live chunk number) % ID_SLOTS
         const uint32_t id_warp = idring + (uint32_t)(quad * 32) * ID_ROW_BYTES;   // slot 0, the warp's first row
+        // int32 output, 128-wide tiles: per-warp staging tile behind the (possibly unused) identity ring
+        const uint32_t i32_tile = idring + (uint32_t)quad * I32_TILE_BYTES;     // (shares the place of the module's ring)
         int pf_ti = 0, pf_ch = 0, pf_slot = 0, cur_slot = 0;
         auto prefetch_next = [&]() {
             bool queued = false;
@@ -267,6 +271,23 @@ conv_tc_i8_kernel(const ConvProblem p, const int ktab_words)
                         cp_async_wait<ID_AHEAD>();                    // this chunk's copy has landed
                         words[ch] = module_chunk(p, dot, id_warp + (uint32_t)cur_slot * (BM * ID_ROW_BYTES), (long)em - lane, n0 + col0, lane);
                         if (++cur_slot == ID_SLOTS) cur_slot = 0;
+                    } else if (BN == 128 && (p.C_out & 3) == 0 && (n0 + col0 + 32 <= p.C_out)) {
+                        // full chunk (warp-uniform): staged, the warp stores whole 128-byte rows
+                        int o[32];
+#pragma unroll
+                        for (int i4 = 0; i4 < 8; ++i4) {
+                            uint4 cc = ld_shared_v4(c0_addr + 4u * (col0 + 4 * i4));
+                            if (two) {
+                                const uint4 c2 = ld_shared_v4(c1_addr + 4u * (col0 + 4 * i4));
+                                cc.x += c2.x; cc.y += c2.y; cc.z += c2.z; cc.w += c2.w;
+                            }
+                            o[4 * i4 + 0] = (int)(v[4 * i4 + 0] >> 5) + rowc + (int)cc.x;
+                            o[4 * i4 + 1] = (int)(v[4 * i4 + 1] >> 5) + rowc + (int)cc.y;
+                            o[4 * i4 + 2] = (int)(v[4 * i4 + 2] >> 5) + rowc + (int)cc.z;
+                            o[4 * i4 + 3] = (int)(v[4 * i4 + 3] >> 5) + rowc + (int)cc.w;
+                        }
+                        const long row0 = (long)em - lane;
+                        store_int32_block(static_cast<int32_t *>(p.out) + row0 * p.C_out + n0 + col0, p.C_out, o, i32_tile, row0, p.M, lane);
                     } else if (em < p.M) {
                         int32_t *dst = static_cast<int32_t *>(p.out) + (long)em * p.C_out + n0 + col0;
                         const bool vec = (p.C_out & 3) == 0 && (n0 + col0 + 32 <= p.C_out);
@@ -488,7 +509,7 @@ int launch_bn(const ConvProblem &p0, cudaStream_t stream)
     if (total >= (1L << 31)) return BCNN_ERR_UNSUPPORTED;
     const unsigned grid = (unsigned)(total < sms ? total : sms);
     const int ktw = ktab_words_for(p);
-    const int smem = smem_bytes<BN>(ktw, p.mode == 2);
+    const int smem = smem_bytes<BN>(ktw, p.mode);
     if (smem > MAX_SMEM) return BCNN_ERR_UNSUPPORTED;
     void (*k)(const ConvProblem, const int) = p.mode == 2 ? conv_tc_i8_kernel<BN, 2> : (p.mode == 1 ? conv_tc_i8_kernel<BN, 1> : conv_tc_i8_kernel<BN, 0>);
     // the attribute is a property of the kernel, not of the launch: always the limit, so that a captured
@@ -516,7 +537,8 @@ int launch_conv_tc_i8(const ConvProblem &p, cudaStream_t stream)
     // 256-wide tiles have a single accumulator buffer (tensor memory also holds the activation
     // ring), so their epilogue is not overlapped: worth it only when the K loop is long
     // (the module epilogue's staging ring only fits beside the 128-wide tiles' weight ring)
-    if (p.C_out > 128 && p.kwords >= 24 && p.mode != 2) {
+    // (int32 output up to K = 4608: the 128-wide tiles' staged stores, whole 128-byte rows, outweigh their extra expansion)
+    if (p.C_out > 128 && p.kwords >= 24 && p.mode != 2 && !(p.mode == 0 && p.kwords <= 144)) {
         // ... unless the narrower tiles fill the last wave so much better that they win anyway: a 128-wide tile
         // costs about 0.6 of a 256-wide one (measured on the K = 2304 and K = 4608 layers)
         int dev = 0, sms = 148;

@@ -74,7 +74,7 @@ struct WsLayout {
 };
 
 template <int BN, int G, bool DUAL, int TEAMS = 1>
-__host__ __device__ inline WsLayout ws_layout(int kwords, bool module)
+__host__ __device__ inline WsLayout ws_layout(int kwords, int mode)
 {
     using C = Cfg<BN, G, DUAL, TEAMS>;
     WsLayout l;
@@ -86,7 +86,8 @@ __host__ __device__ inline WsLayout ws_layout(int kwords, bool module)
     l.row_kt = (l.ktiles <= 3 && C::STAGES >= (G - 1) * l.ktiles + 1) ? l.ktiles : 0;
     l.bits_bytes = C::BITS_BYTES * (l.row_kt ? l.row_kt : 1);
     l.smem = 1024 + l.ktiles * C::W_TILE_BYTES + l.bits_bytes + BN * 4 + l.ktiles * 32;
-    if (module) l.smem += TEAMS * ID_RING_BYTES + 16;         // identity staging rings of the module epilogue
+    if (mode == 2) l.smem += TEAMS * ID_RING_BYTES + 16;      // identity staging rings of the module epilogue
+    if (mode == 0) l.smem += TEAMS * EPI_WARPS * I32_TILE_BYTES + 16;   // store staging tiles of the int32 epilogue
     // Tensor memory is shared out by the resident CTAs (all 512 columns, or 256 each for two): ask
     // for enough shared memory that no further CTA of this kernel fits on the SM (it would sit in
     // tcgen05.alloc until a neighbour exits).
@@ -113,7 +114,7 @@ conv_tc_ws_kernel(const ConvProblem p)
 
     const int tid = threadIdx.x;
     const int warp = tid >> 5, lane = tid & 31;
-    const WsLayout L = ws_layout<BN, G, DUAL, TEAMS>(p.kwords, MODULE);
+    const WsLayout L = ws_layout<BN, G, DUAL, TEAMS>(p.kwords, MODE);
     const int ktiles = L.ktiles;
     constexpr int STAGES = C::STAGES;
     const int m_tiles = (p.M + BM - 1) / BM;
@@ -255,6 +256,7 @@ conv_tc_ws_kernel(const ConvProblem p)
         const int quad = warp & 3;
         const int erow = quad * 32 + lane;
         const int team = (warp - 1) >> 2;                        // takes the tiles team, team + TEAMS, ...
+        const uint32_t i32_tile = idring + (uint32_t)(team * EPI_WARPS + quad) * I32_TILE_BYTES;   // int32 epilogue (shares the place of the module's rings)
         bool alive = true;
         // module epilogue: chunk q of this thread's row sequence = (tile q / nch, chunk q % nch); its identity values
         // are staged ID_AHEAD chunks ahead in ring slot q % ID_SLOTS
@@ -316,6 +318,19 @@ conv_tc_ws_kernel(const ConvProblem p)
                         cp_async_wait<ID_AHEAD>();                    // this chunk's copy has landed
                         words[ch] = module_chunk(p, dot, id_warp + (uint32_t)cur_slot * (BM * ID_ROW_BYTES), (long)em - lane, n0 + col0, lane);
                         if (++cur_slot == ID_SLOTS) cur_slot = 0;
+                    } else if ((p.C_out & 3) == 0 && (n0 + col0 + 32 <= p.C_out)) {
+                        // full chunk (warp-uniform): staged, the warp stores whole 128-byte rows
+                        int o[32];
+#pragma unroll
+                        for (int i4 = 0; i4 < 8; ++i4) {
+                            const uint4 cc = ld_shared_v4(colc_addr + 4u * (col0 + 4 * i4));
+                            o[4 * i4 + 0] = ((int)v[4 * i4 + 0] >> 5) + (int)cc.x;
+                            o[4 * i4 + 1] = ((int)v[4 * i4 + 1] >> 5) + (int)cc.y;
+                            o[4 * i4 + 2] = ((int)v[4 * i4 + 2] >> 5) + (int)cc.z;
+                            o[4 * i4 + 3] = ((int)v[4 * i4 + 3] >> 5) + (int)cc.w;
+                        }
+                        const long row0 = (long)em - lane;
+                        store_int32_block(static_cast<int32_t *>(p.out) + row0 * p.C_out + n0 + col0, p.C_out, o, i32_tile, row0, p.M, lane);
                     } else if (em < p.M) {
                         int32_t *dst = static_cast<int32_t *>(p.out) + (long)em * p.C_out + n0 + col0;
                         const bool vec = (p.C_out & 3) == 0 && (n0 + col0 + 32 <= p.C_out);
@@ -522,7 +537,7 @@ int launch_ws(const ConvProblem &p0, cudaStream_t stream)
     cudaGetDevice(&dev);
     cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     using C = Cfg<BN, G, DUAL, TEAMS>;
-    const WsLayout L = ws_layout<BN, G, DUAL, TEAMS>(p.kwords, p.mode == 2);
+    const WsLayout L = ws_layout<BN, G, DUAL, TEAMS>(p.kwords, p.mode);
     const long m_tiles = ((long)p.M + BM - 1) / BM;
     const long slots = (long)sms * C::CTAS_PER_SM;
     const long n_tiles = (p.C_out + BN - 1) / BN;
@@ -544,7 +559,7 @@ int launch_ws(const ConvProblem &p0, cudaStream_t stream)
 template <int BN, int G, bool DUAL, int TEAMS = 1>
 bool fits(const ConvProblem &p)
 {
-    return ws_layout<BN, G, DUAL, TEAMS>(p.kwords, p.mode == 2).smem <= (DUAL ? 113 * 1024 : MAX_SMEM - 1024);
+    return ws_layout<BN, G, DUAL, TEAMS>(p.kwords, p.mode).smem <= (DUAL ? 113 * 1024 : MAX_SMEM - 1024);
 }
 
 }  // namespace

@@ -417,6 +417,30 @@ __device__ __forceinline__ void gather_stage(const uint32_t *x, const RowCursor 
     }
 }
 
+// int32 output of one accumulator chunk: 32 rows (one per lane) x 32 consecutive columns.  A lane storing its own
+// row touches 32 rows x 16 bytes per instruction; staged through shared memory the warp stores 4 rows x 128
+// contiguous bytes per instruction instead.  `warp_tile`: I32_TILE_BYTES of shared memory owned by this warp;
+// `dst0` points at (row0, first column), `ldc` is the row pitch in elements (a multiple of 4, 16-byte aligned rows).
+// All 32 lanes must call it.
+constexpr int I32_ROW_BYTES = 144;                         // 128 + 16: conflict-free both ways
+constexpr int I32_TILE_BYTES = 32 * I32_ROW_BYTES;
+__device__ __forceinline__ void store_int32_block(int32_t *dst0, long ldc, const int (&o)[32], uint32_t warp_tile,
+                                                  long row0, long M, int lane)
+{
+    const uint32_t mine = warp_tile + (uint32_t)(lane * I32_ROW_BYTES);
+#pragma unroll
+    for (int i4 = 0; i4 < 8; ++i4)
+        st_shared_v4(mine + 16u * i4, (uint32_t)o[4 * i4], (uint32_t)o[4 * i4 + 1], (uint32_t)o[4 * i4 + 2], (uint32_t)o[4 * i4 + 3]);
+    __syncwarp();
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        const int r = (lane >> 3) + 4 * i;
+        const uint4 v = ld_shared_v4(warp_tile + (uint32_t)(r * I32_ROW_BYTES + (lane & 7) * 16));
+        if (row0 + r < M) *reinterpret_cast<uint4 *>(dst0 + (long)r * ldc + 4 * (lane & 7)) = v;
+    }
+    __syncwarp();
+}
+
 // Convolution-module epilogue (Section 4.2.1).
 //
 // Identity staging: an epilogue thread owns one output row and walks its 32-channel chunks in order.  The 64 bytes of
