@@ -482,16 +482,14 @@ __device__ __forceinline__ void module_prefetch(const ConvProblem &p, uint32_t w
 // same slot, from where the warp stores them cooperatively (same 8 rows x 64 bytes per instruction), and returns
 // the 32 sign bits of the lane's row (bit i = channel n0 + i).  The channel count is a multiple of 32, so every
 // 8-channel group is 16-byte aligned.  All 32 lanes must call it.
-__device__ __forceinline__ uint32_t module_chunk(const ConvProblem &p, const int (&dot)[32], uint32_t warp_slot,
-                                                 long row0, int n0, int lane)
+template <bool HAS_ID, bool HAS_NB>
+__device__ __forceinline__ uint32_t module_chunk_t(const ConvProblem &p, const int (&dot)[32], uint32_t slot_addr, int n0)
 {
     uint32_t bits = 0;
-    const uint32_t slot_addr = warp_slot + (uint32_t)(lane * ID_ROW_BYTES);
-    __syncwarp();                                           // the cooperative copies of all lanes have landed
 #pragma unroll
     for (int g = 0; g < 4; ++g) {                           // 8 channels per group
         uint4 idv = make_uint4(0u, 0u, 0u, 0u);
-        if (p.identity) idv = ld_shared_v4(slot_addr + 16u * g);
+        if (HAS_ID) idv = ld_shared_v4(slot_addr + 16u * g);
         const uint32_t idw[4] = {idv.x, idv.y, idv.z, idv.w};
         uint32_t ow[4];
 #pragma unroll
@@ -501,29 +499,40 @@ __device__ __forceinline__ uint32_t module_chunk(const ConvProblem &p, const int
             const float4 sh = __ldg(reinterpret_cast<const float4 *>(p.bn_shift + n));
             const float4 sl = __ldg(reinterpret_cast<const float4 *>(p.slope + n));
             float4 nb = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (p.next_bias) nb = __ldg(reinterpret_cast<const float4 *>(p.next_bias + n));
+            if (HAS_NB) nb = __ldg(reinterpret_cast<const float4 *>(p.next_bias + n));
             const float scs[4] = {sc.x, sc.y, sc.z, sc.w}, shs[4] = {sh.x, sh.y, sh.z, sh.w};
             const float sls[4] = {sl.x, sl.y, sl.z, sl.w}, nbs[4] = {nb.x, nb.y, nb.z, nb.w};
-            unsigned short hv[4];
 #pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                const int c = 8 * g + 4 * h + e;
-                const uint32_t pair = idw[2 * h + (e >> 1)];
-                const __half idh = __ushort_as_half((unsigned short)((e & 1) ? (pair >> 16) : (pair & 0xFFFFu)));
-                float t = __fmul_rn(__int2float_rn(dot[c]), scs[e]);
-                t = __fadd_rn(t, shs[e]);
-                const float u = p.identity ? __fadd_rn(t, __half2float(idh)) : t;
-                const float r = (u >= 0.0f) ? u : __fmul_rn(sls[e], u);
-                const __half y = __float2half_rn(r);
-                hv[e] = __half_as_ushort(y);
-                const float sv = __fadd_rn(__half2float(y), nbs[e]);
-                bits |= (sv >= 0.0f ? 1u : 0u) << c;
+            for (int q = 0; q < 2; ++q) {                   // two channels at a time: paired fp16 <-> fp32 conversions
+                const int c = 8 * g + 4 * h + 2 * q;
+                const float2 idf = __half22float2(*reinterpret_cast<const __half2 *>(&idw[2 * h + q]));
+                float r[2];
+#pragma unroll
+                for (int e = 0; e < 2; ++e) {
+                    float t = __fmul_rn(__int2float_rn(dot[c + e]), scs[2 * q + e]);
+                    t = __fadd_rn(t, shs[2 * q + e]);
+                    const float u = HAS_ID ? __fadd_rn(t, e ? idf.y : idf.x) : t;
+                    r[e] = (u >= 0.0f) ? u : __fmul_rn(sls[2 * q + e], u);
+                }
+                const __half2 y2 = __floats2half2_rn(r[0], r[1]);      // round to nearest even, element-wise
+                ow[2 * h + q] = *reinterpret_cast<const uint32_t *>(&y2);
+                const float2 yf = __half22float2(y2);
+                bits |= (__fadd_rn(yf.x, nbs[2 * q]) >= 0.0f ? 1u : 0u) << c;
+                bits |= (__fadd_rn(yf.y, nbs[2 * q + 1]) >= 0.0f ? 1u : 0u) << (c + 1);
             }
-            ow[2 * h] = (uint32_t)hv[0] | ((uint32_t)hv[1] << 16);
-            ow[2 * h + 1] = (uint32_t)hv[2] | ((uint32_t)hv[3] << 16);
         }
         st_shared_v4(slot_addr + 16u * g, ow[0], ow[1], ow[2], ow[3]);
     }
+    return bits;
+}
+__device__ __forceinline__ uint32_t module_chunk(const ConvProblem &p, const int (&dot)[32], uint32_t warp_slot,
+                                                 long row0, int n0, int lane)
+{
+    const uint32_t slot_addr = warp_slot + (uint32_t)(lane * ID_ROW_BYTES);
+    __syncwarp();                                           // the cooperative copies of all lanes have landed
+    uint32_t bits;
+    if (p.identity) bits = p.next_bias ? module_chunk_t<true, true>(p, dot, slot_addr, n0) : module_chunk_t<true, false>(p, dot, slot_addr, n0);
+    else bits = p.next_bias ? module_chunk_t<false, true>(p, dot, slot_addr, n0) : module_chunk_t<false, false>(p, dot, slot_addr, n0);
     __syncwarp();                                           // the rows of all lanes are staged
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
