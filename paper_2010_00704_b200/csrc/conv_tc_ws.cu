@@ -47,22 +47,21 @@ constexpr int ERR_EPILOGUE_TIMEOUT = 113;
 // bound by the epilogue warps.
 template <int BN, int G, bool DUAL, int TEAMS = 1> struct Cfg {
     static constexpr int FIRST_PRODUCER_THREAD = 32 * (1 + EPI_WARPS * TEAMS);
-    static constexpr int BNX = BN;
     static constexpr int PROD_THREADS = G * BM;
-    // Tensor memory (512 columns): NBUF accumulator buffers of BNX columns, then the activation ring,
+    // Tensor memory (512 columns): NBUF accumulator buffers of BN columns, then the activation ring,
     // one stage = 128 rows x 128 expanded bytes = 32 columns.
     static constexpr int TMEM_COLS = DUAL ? 256 : 512;
     static constexpr int NBUF = DUAL ? (BN == 128 ? 1 : 2) : (BN == 32 ? 4 : (BN == 64 ? 3 : 2));
     static constexpr int CONTROL_WARP = (FIRST_PRODUCER_THREAD + PROD_THREADS) / 32;
     static constexpr int THREADS = FIRST_PRODUCER_THREAD + PROD_THREADS + 32;
-    static constexpr int A_COL0 = NBUF * BNX;
+    static constexpr int A_COL0 = NBUF * BN;
     static constexpr int STAGES = (TMEM_COLS - A_COL0) / 32 > 8 ? 8 : (TMEM_COLS - A_COL0) / 32;
     static constexpr int CTAS_PER_SM = DUAL ? 2 : 1;
     // registers are granted in blocks of 8 per thread: bound the pair of CTAs to 64 registers per thread
     static constexpr int BOUND_THREADS = DUAL ? 512 : THREADS;
     static_assert(A_COL0 + STAGES * 32 <= TMEM_COLS, "tensor memory budget");
     static_assert(STAGES >= G, "a producer group must not lap the ring (parity waits)");
-    static constexpr int W_TILE_BYTES = BNX * ROWB;           // one K stage of the expanded weights
+    static constexpr int W_TILE_BYTES = BN * ROWB;           // one K stage of the expanded weights
     static constexpr int BITS_BYTES = PF * PROD_THREADS * 16;
 };
 
@@ -103,7 +102,6 @@ conv_tc_ws_kernel(const ConvProblem p)
     using C = Cfg<BN, G, DUAL, TEAMS>;
     static_assert(C::NBUF % TEAMS == 0, "a team's tiles must map to a fixed set of accumulator buffers");
     constexpr bool FUSED = MODE == 1, MODULE = MODE == 2;
-    constexpr int BNX = C::BNX;
     constexpr int NBUF = C::NBUF;
     constexpr int MAX_STAGES = 8;
 
@@ -129,7 +127,7 @@ conv_tc_ws_kernel(const ConvProblem p)
     const int total_items = my_tiles * ktiles;
 
     // shared-memory map (all 1024-byte aligned where the MMA reads)
-    const uint32_t wexp = (smem_u32(smem_raw) + 1023u) & ~1023u;          // [ktiles][BNX rows][128 B]
+    const uint32_t wexp = (smem_u32(smem_raw) + 1023u) & ~1023u;          // [ktiles][BN rows][128 B]
     const uint32_t bits_ring = wexp + (uint32_t)ktiles * C::W_TILE_BYTES; // [PF][PROD_THREADS][16 B]
     const uint32_t colc_addr = bits_ring + (uint32_t)L.bits_bytes;                 // [BN] int32
     const uint32_t ktab_addr = colc_addr + BN * 4;                        // unit table: [ktiles * 4 / gw] x {word offset, tap bit}
@@ -200,7 +198,7 @@ conv_tc_ws_kernel(const ConvProblem p)
         // stage at a time through named barrier 1 + slot.  There is one issuer on purpose: the
         // producers' parity waits rely on the ring being consumed in order (a second issuer working on
         // the next tile lets a late slot fall two phases behind a waiting producer).
-        constexpr uint32_t idesc = make_idesc(BNX) | (1u << 10);                  // B operand: signed bytes
+        constexpr uint32_t idesc = make_idesc(BN) | (1u << 10);                  // B operand: signed bytes
         const uint64_t desc0 = make_desc(0);
         const uint32_t desc_hi = (uint32_t)(desc0 >> 32);
         const uint32_t tmem_u = __shfl_sync(0xffffffffu, tmem_base, 0);             // warp-uniform copy for the issuer
@@ -208,7 +206,7 @@ conv_tc_ws_kernel(const ConvProblem p)
         const uint32_t b_lo0 = (uint32_t)desc0 | ((wexp & 0x3FFFFu) >> 4);       // + kt * (W_TILE_BYTES / 16)
         int s = 0, buf = 0;
         for (int ti = 0; ti < my_tiles; ++ti) {
-            const uint32_t d_tmem = tmem_u + (uint32_t)(buf * BNX);
+            const uint32_t d_tmem = tmem_u + (uint32_t)(buf * BN);
             const uint32_t tfull = tfull_bar(buf);
             for (int kt = 0; kt < ktiles; ++kt) {
                 const uint32_t a_t = a_tmem0 + (uint32_t)s * 32u;
@@ -284,7 +282,7 @@ conv_tc_ws_kernel(const ConvProblem p)
             alive = __all_sync(0xffffffffu, alive && !*abort_flag);
             if (!alive) break;
             tc_fence_after();
-            const uint32_t t_addr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(buf * BNX);
+            const uint32_t t_addr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(buf * BN);
             uint32_t words[BN / 32];
 #pragma unroll
             for (int ch = 0; ch < BN / 32; ++ch) {
