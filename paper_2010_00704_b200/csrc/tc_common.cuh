@@ -333,6 +333,7 @@ struct TileStep {
     uint32_t rows;
     int db, doh, dow;
     uint32_t pat;            // bit r*kw for every kernel row r
+    bool pointwise;          // 1x1, stride 1, no padding: row m reads input pixel m, no coordinates needed
 };
 __device__ __forceinline__ TileStep make_tile_step(const ConvProblem &p, uint32_t rows)
 {
@@ -345,6 +346,7 @@ __device__ __forceinline__ TileStep make_tile_step(const ConvProblem &p, uint32_
     s.dow = (int)(rem - (uint32_t)s.doh * (uint32_t)p.OW);
     s.pat = 0;
     for (int r = 0; r < p.kh; ++r) s.pat |= 1u << (r * p.kw);
+    s.pointwise = p.kh == 1 && p.kw == 1 && p.stride == 1 && p.pad == 0;
     return s;
 }
 struct RowCursor {
@@ -364,6 +366,7 @@ __device__ __forceinline__ void row_locate(const ConvProblem &p, RowCursor &rc)
 __device__ __forceinline__ void row_step(const ConvProblem &p, const TileStep &s, RowCursor &rc)
 {
     rc.m += s.rows;
+    if (s.pointwise) return;
     rc.ow += s.dow;
     if (rc.ow >= p.OW) { rc.ow -= p.OW; ++rc.oh; }
     rc.oh += s.doh;
@@ -373,6 +376,11 @@ __device__ __forceinline__ void row_step(const ConvProblem &p, const TileStep &s
 __device__ __forceinline__ uint32_t low_bits(int n) { return (1u << n) - 1u; }   // 0 <= n <= 31
 __device__ __forceinline__ void row_window(const ConvProblem &p, const TileStep &s, RowCursor &rc)
 {
+    if (s.pointwise) {                                      // warp-uniform
+        rc.base = (int)(rc.m * (uint32_t)p.cw);
+        rc.mask = rc.m < (uint32_t)p.M ? 1u : 0u;
+        return;
+    }
     const int ih0 = rc.oh * p.stride - p.pad, iw0 = rc.ow * p.stride - p.pad;
     rc.base = ((rc.b * p.H + ih0) * p.W + iw0) * p.cw;
     // taps t with 0 <= iw0 + t < W and r with 0 <= ih0 + r < H (an empty range gives an empty mask)
