@@ -8,7 +8,10 @@
 // Every product with a set activation bit is +-64, accumulators are int32 in tensor memory, and with
 // S = sum over set activation bits of the weight signs (acc = 64 S):
 //   sum a*g = 2 S + K - 2 popc(G)          (a, g in {-1,+1})
-// so the epilogue needs one constant per output channel and nothing per row.
+// so the epilogue needs one constant per output channel and nothing per row - and not even an addition: the
+// accumulator buffers START from that constant (scaled by 32; the threshold folded in for the packed output).  The
+// epilogue team writes the constants into its buffers once, and again right after reading a tile out of one; every
+// MMA accumulates.  The packed output is then the complement of the accumulators' sign bits.
 // Differences to conv_tc_i8.cu, all aimed at short tiles (a 128 x 32 x 32 tile is one MMA instruction):
 //   * the CTA expands its weight tile ONCE into shared memory and keeps it for all its
 //     output tiles; only activations stream through the ring;
@@ -172,14 +175,17 @@ conv_tc_ws_kernel(const ConvProblem p)
         int pop = 0;
         if (c < cn)
             for (int kw = 0; kw < p.kwords; ++kw) pop += __popc(__ldg(p.w + (long)(n0 + c) * p.kwords + kw));
-        // with acc = 64 * S:   int32: (acc >> 5) + (K - 2*pop)      fused: acc + 32*(K - 2*pop - thr) >= 0
+        // The accumulators start from a per-channel constant instead of zero (the epilogue writes it back after
+        // reading a buffer, every MMA accumulates), so with acc = 64 * S + cst:
+        //   int32: acc >> 5 with cst = 32 * (K - 2*pop)        fused: acc >= 0 with cst = 32 * (K - 2*pop - thr)
         // (a threshold beyond +-(K + 1) decides like that bound; clamping keeps the constant inside int32)
         int cst = p.K - 2 * pop;
         if (FUSED) {
             int t = c < cn ? __ldg(p.thr + n0 + c) : 0;
             t = max(min(t, p.K + 1), -p.K - 1);
-            cst = 32 * (cst - t);
+            cst -= t;
         }
+        cst *= 32;
         asm volatile("st.shared.b32 [%0], %1;" ::"r"(colc_addr + 4u * c), "r"(cst) : "memory");
     }
     const int gw = gather_width(p.cw);
@@ -217,7 +223,7 @@ conv_tc_ws_kernel(const ConvProblem p)
                 tc_fence_after();
                 // per 32 bytes of K: 8 tensor-memory columns of A, +2 (16-byte units) in the B descriptor
                 if (elect_one()) {
-                    tc_mma_i8_ts(d_tmem, a_t, b_lo, desc_hi, idesc, kt > 0 ? 1u : 0u);
+                    tc_mma_i8_ts(d_tmem, a_t, b_lo, desc_hi, idesc, 1u);      // always accumulates: the buffer holds the constants
                     if (nk > 1) tc_mma_i8_ts(d_tmem, a_t + 8u, b_lo + 2u, desc_hi, idesc, 1u);
                     if (nk > 2) tc_mma_i8_ts(d_tmem, a_t + 16u, b_lo + 4u, desc_hi, idesc, 1u);
                     if (nk > 3) tc_mma_i8_ts(d_tmem, a_t + 24u, b_lo + 6u, desc_hi, idesc, 1u);
@@ -237,7 +243,7 @@ conv_tc_ws_kernel(const ConvProblem p)
         // After a time-out the remaining stages are released without waiting so that the issuer,
         // whose barrier wait has no time limit, always terminates; the error word tells the host.
         int s = 0, buf = 0;
-        uint32_t ring_phase = 0, buf_phase = 1;      // first use of every accumulator buffer: free
+        uint32_t ring_phase = 0, buf_phase = 0;      // every accumulator buffer is handed over by its epilogue team, first after initialising it
         bool alive = true;
         for (int ti = 0; ti < my_tiles; ++ti) {
             if (lane == 0 && alive) alive = mbar_wait(tempty_bar(buf), buf_phase, abort_flag, p.err, ERR_MMA_TIMEOUT);
@@ -273,6 +279,27 @@ conv_tc_ws_kernel(const ConvProblem p)
         };
         if (MODULE)
             for (int a = 0; a < ID_AHEAD; ++a) prefetch_next();
+        // write the per-channel constants into 32 accumulator columns of this warp's rows (8 columns at a time:
+        // the values are the same for every row)
+        auto write_consts = [&](uint32_t t_chunk, int col0) {
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const uint4 a = ld_shared_v4(colc_addr + 4u * (col0 + 8 * q)), b = ld_shared_v4(colc_addr + 4u * (col0 + 8 * q + 4));
+                const uint32_t c8[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
+                tc_st8_nowait(t_chunk + 8u * q, c8);
+            }
+        };
+        // the team's accumulator buffers start out holding the constants
+        for (int b = team; b < NBUF; b += TEAMS) {
+            const uint32_t tb = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(b * BN);
+#pragma unroll
+            for (int ch = 0; ch < BN / 32; ++ch)
+                if (ch * 32 < cn) write_consts(tb + (uint32_t)(ch * 32), ch * 32);
+            tc_wait_st();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(tempty_bar(b));
+        }
         for (int ti = team; ti < my_tiles; ti += TEAMS) {
             const int buf = ti % NBUF;                            // tiles use the accumulator buffers in turn
             const uint32_t buf_phase = (uint32_t)(ti / NBUF) & 1u;
@@ -291,27 +318,17 @@ conv_tc_ws_kernel(const ConvProblem p)
                 if (col0 < cn) {                                      // warp-uniform
                     uint32_t v[32];
                     tc_ld32(t_addr + (uint32_t)col0, v);
+                    write_consts(t_addr + (uint32_t)col0, col0);      // the buffer's next tile starts from the constants again
                     if (FUSED) {
+                        // bit = (v >= 0): the sign bits are shifted in, last column first
                         uint32_t acc = 0;
 #pragma unroll
-                        for (int i4 = 7; i4 >= 0; --i4) {
-                            const uint4 cc = ld_shared_v4(colc_addr + 4u * (col0 + 4 * i4));
-                            acc = __funnelshift_l((uint32_t)((int)v[4 * i4 + 3] + (int)cc.w), acc, 1);
-                            acc = __funnelshift_l((uint32_t)((int)v[4 * i4 + 2] + (int)cc.z), acc, 1);
-                            acc = __funnelshift_l((uint32_t)((int)v[4 * i4 + 1] + (int)cc.y), acc, 1);
-                            acc = __funnelshift_l((uint32_t)((int)v[4 * i4 + 0] + (int)cc.x), acc, 1);
-                        }
+                        for (int i = 31; i >= 0; --i) acc = __funnelshift_l(v[i], acc, 1);
                         words[ch] = ~acc;
                     } else if (MODULE) {
                         int dot[32];
 #pragma unroll
-                        for (int i4 = 0; i4 < 8; ++i4) {
-                            const uint4 cc = ld_shared_v4(colc_addr + 4u * (col0 + 4 * i4));
-                            dot[4 * i4 + 0] = ((int)v[4 * i4 + 0] >> 5) + (int)cc.x;
-                            dot[4 * i4 + 1] = ((int)v[4 * i4 + 1] >> 5) + (int)cc.y;
-                            dot[4 * i4 + 2] = ((int)v[4 * i4 + 2] >> 5) + (int)cc.z;
-                            dot[4 * i4 + 3] = ((int)v[4 * i4 + 3] >> 5) + (int)cc.w;
-                        }
+                        for (int i = 0; i < 32; ++i) dot[i] = (int)v[i] >> 5;
                         prefetch_next();
                         cp_async_wait<ID_AHEAD>();                    // this chunk's copy has landed
                         words[ch] = module_chunk(p, dot, id_warp + (uint32_t)cur_slot * (BM * ID_ROW_BYTES), (long)em - lane, n0 + col0, lane);
@@ -320,13 +337,7 @@ conv_tc_ws_kernel(const ConvProblem p)
                         // full chunk (warp-uniform): staged, the warp stores whole 128-byte rows
                         int o[32];
 #pragma unroll
-                        for (int i4 = 0; i4 < 8; ++i4) {
-                            const uint4 cc = ld_shared_v4(colc_addr + 4u * (col0 + 4 * i4));
-                            o[4 * i4 + 0] = ((int)v[4 * i4 + 0] >> 5) + (int)cc.x;
-                            o[4 * i4 + 1] = ((int)v[4 * i4 + 1] >> 5) + (int)cc.y;
-                            o[4 * i4 + 2] = ((int)v[4 * i4 + 2] >> 5) + (int)cc.z;
-                            o[4 * i4 + 3] = ((int)v[4 * i4 + 3] >> 5) + (int)cc.w;
-                        }
+                        for (int i = 0; i < 32; ++i) o[i] = (int)v[i] >> 5;
                         const long row0 = (long)em - lane;
                         store_int32_block(static_cast<int32_t *>(p.out) + row0 * p.C_out + n0 + col0, p.C_out, o, i32_tile, row0, p.M, lane);
                     } else if (em < p.M) {
@@ -334,12 +345,11 @@ conv_tc_ws_kernel(const ConvProblem p)
                         const bool vec = (p.C_out & 3) == 0 && (n0 + col0 + 32 <= p.C_out);
 #pragma unroll
                         for (int i4 = 0; i4 < 8; ++i4) {
-                            const uint4 cc = ld_shared_v4(colc_addr + 4u * (col0 + 4 * i4));
                             int4 o;
-                            o.x = ((int)v[4 * i4 + 0] >> 5) + (int)cc.x;
-                            o.y = ((int)v[4 * i4 + 1] >> 5) + (int)cc.y;
-                            o.z = ((int)v[4 * i4 + 2] >> 5) + (int)cc.z;
-                            o.w = ((int)v[4 * i4 + 3] >> 5) + (int)cc.w;
+                            o.x = (int)v[4 * i4 + 0] >> 5;
+                            o.y = (int)v[4 * i4 + 1] >> 5;
+                            o.z = (int)v[4 * i4 + 2] >> 5;
+                            o.w = (int)v[4 * i4 + 3] >> 5;
                             if (vec) {
                                 *reinterpret_cast<int4 *>(dst + 4 * i4) = o;
                             } else {
@@ -353,6 +363,7 @@ conv_tc_ws_kernel(const ConvProblem p)
                     }
                 }
             }
+            tc_wait_st();                     // the constants are back in the buffer
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(tempty_bar(buf));
