@@ -33,7 +33,7 @@ from paper_2010_00704_b200 import synth, workloads as wl  # noqa: E402
 
 # DRAM bytes (read + write) per launch of the roofline's launch, from the ncu capture summarised under
 # profiles/; None until a capture of the current kernel exists.
-ROOFLINE_TRAFFIC = {"L2_3x3s2_32": 51865088}
+ROOFLINE_TRAFFIC = {"L2_3x3s2_32": 51889920}
 POPC_PEAK_TOPS = 385.0
 
 METRIC = "binary conv throughput (2*M*N*K bit-ops/s), backbone-shaped stack"
