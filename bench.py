@@ -31,11 +31,6 @@ if ROOT not in sys.path:
 
 from paper_2010_00704_b200 import synth, workloads as wl  # noqa: E402
 
-# DRAM bytes (read + write) per launch of the roofline's launch, from the ncu capture summarised under
-# profiles/; None until a capture of the current kernel exists.
-ROOFLINE_TRAFFIC = {"L2_3x3s2_32": 51889920}
-POPC_PEAK_TOPS = 385.0
-
 METRIC = "binary conv throughput (2*M*N*K bit-ops/s), backbone-shaped stack"
 UNIT = "TOPS"
 WORKLOAD = "backbone18 @ batch 256: 224x224x4 fp32 -> pack(32ch) -> 18 fused binary conv layers (pack + layer 1 in one kernel)"
@@ -156,6 +151,19 @@ def oracle_backbone_seconds(n_images: int, x, bias, ws, ts):
     return time.perf_counter() - t0
 
 
+def checker_backbone_seconds(n_images: int, x, bias, ws, ts):
+    """Time the bit-packed CPU checker (xor + popcount loops; not the oracle) on the first n_images images."""
+    import oracle
+    layers = wl.BACKBONE18
+    _, _, _, R = wl.BACKBONE18_INPUT
+    cur = synth.pack_bits(oracle.binarize(x[:n_images], bias, R))       # untimed: the checker starts from packed bits
+    t0 = time.perf_counter()
+    for l, w, t in zip(layers, ws, ts):
+        acc = oracle.checker_conv2d(cur, w, (n_images, l.H, l.W, l.C_in, l.C_out, l.k, l.k), l.stride, l.pad)
+        cur = synth.pack_bits(np.where(acc >= t, 1, -1).astype(np.int8))
+    return time.perf_counter() - t0
+
+
 def cpu_baseline(target_seconds: float = 15.0):
     import oracle
     oracle.build()
@@ -165,9 +173,15 @@ def cpu_baseline(target_seconds: float = 15.0):
     n = int(max(1, min(cap, target_seconds / max(t1, 1e-3))))
     secs = oracle_backbone_seconds(n, x, bias, ws, ts)
     ops = wl.chain_ops(wl.BACKBONE18, n)
+    c1 = checker_backbone_seconds(2, x, bias, ws, ts) / 2
+    nc = int(max(1, min(cap, 5.0 / max(c1, 1e-3))))
+    csecs = checker_backbone_seconds(nc, x, bias, ws, ts)
     return {"value": ops / secs / 1e12, "unit": UNIT, "cores": oracle.threads(), "kind": "oracle",
             "sample": f"first {n} images of the batch through pack + 18 layers ({secs:.1f} s)",
-            "images_per_s": n / secs}
+            "images_per_s": n / secs,
+            "packed_checker": {"value": wl.chain_ops(wl.BACKBONE18, nc) / csecs / 1e12, "unit": UNIT, "cores": oracle.threads(),
+                               "kind": "bit-packed xor + popcount loops (the tests' full-coverage checker, not the oracle)",
+                               "sample": f"first {nc} images through the 18 layers ({csecs:.1f} s)", "images_per_s": nc / csecs}}
 
 
 def run_reference(args):
@@ -203,7 +217,155 @@ def run_reference(args):
     return 0
 
 
+# ----------------------------------------------------------------------------- instruction probes
+
+PROBES_SRC = os.path.join(ROOT, "bench_probes.cu")
+PROBES_LIB = os.path.join(ROOT, "bench_probes.so")
+
+
+def build_probes() -> str:
+    """Compile bench_probes.cu (instruction-throughput probes) into bench_probes.so beside this file."""
+    csrc = os.path.join(ROOT, "paper_2010_00704_b200", "csrc")
+    deps = [PROBES_SRC, os.path.join(csrc, "tc_common.cuh"), os.path.join(csrc, "bcnn_common.cuh")]
+    if not os.path.exists(PROBES_LIB) or os.path.getmtime(PROBES_LIB) < max(os.path.getmtime(d) for d in deps):
+        tmp = PROBES_LIB + f".tmp{os.getpid()}"
+        subprocess.run([os.environ.get("NVCC", "nvcc"), "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3",
+                        "-std=c++17", "-shared", "-Xcompiler", "-fPIC", "-I", os.path.join(ROOT, "include"), "-I", csrc,
+                        "-o", tmp, PROBES_SRC, "-lcudart"], check=True)
+        os.replace(tmp, PROBES_LIB)
+    return PROBES_LIB
+
+
+def run_probes():
+    """Instruction peaks measured in this process (TOP/s, 1 MAC = 2 ops); see bench_probes.cu."""
+    import ctypes
+    lib = ctypes.CDLL(build_probes())
+    dbl, i32 = ctypes.c_double, ctypes.c_int
+    out = {}
+    ms, macs, derr = dbl(0), dbl(0), i32(0)
+    for n in (256, 128, 64, 32):
+        st = lib.probe_tcgen05_i8(n, 4000 * (256 // n), ctypes.byref(ms), ctypes.byref(macs), ctypes.byref(derr))
+        if st != 0 or derr.value != 0:
+            raise SystemExit(f"tcgen05 probe failed: status {st}, device error {derr.value}")
+        out[f"tcgen05_i8_n{n}"] = 2 * macs.value / (ms.value / 1e3) / 1e12
+    for mode, name in ((0, "mma_sync_b1_and_popc"), (1, "mma_sync_b1_xor_popc"), (2, "mma_sync_s8")):
+        st = lib.probe_mma_sync(mode, 2000 if mode < 2 else 20000, ctypes.byref(ms), ctypes.byref(macs))
+        if st != 0:
+            raise SystemExit(f"mma.sync probe failed: status {st}")
+        out[name] = 2 * macs.value / (ms.value / 1e3) / 1e12
+    st = lib.probe_popc(20000, ctypes.byref(ms), ctypes.byref(macs))
+    if st != 0:
+        raise SystemExit(f"popc probe failed: status {st}")
+    out["xor_popc"] = 2 * macs.value / (ms.value / 1e3) / 1e12
+    return out
+
+
+def roofline_traffic(summary_name: str, sources):
+    """DRAM bytes per launch from a tracked ncu summary under profiles/ (a line `traffic_bytes_per_launch: N`), or
+    None when there is none or when the kernel's sources changed after the capture (the summary's `source_sha` line
+    is the sha1 of the concatenated source files)."""
+    import hashlib
+    path = os.path.join(ROOT, "profiles", summary_name)
+    if not os.path.exists(path):
+        return None
+    fields = {}
+    for line in open(path):
+        if ":" in line:
+            k, v = line.split(":", 1)
+            fields[k.strip()] = v.strip()
+    h = hashlib.sha1()
+    for src in sources:
+        h.update(open(os.path.join(ROOT, "paper_2010_00704_b200", "csrc", src), "rb").read())
+    if fields.get("source_sha") != h.hexdigest():
+        return None
+    try:
+        return int(fields["traffic_bytes_per_launch"])
+    except (KeyError, ValueError):
+        return None
+
+
 # ----------------------------------------------------------------------------- GPU arm
+
+def timed_launches(fn, steps: int, warmup: int, flush=None):
+    """CUDA-event time of each of `steps` calls of fn (ms), after `warmup` untimed ones; `flush` (a device buffer
+    larger than L2) is overwritten before every timed call."""
+    import torch
+    for _ in range(warmup):
+        fn()
+    ts = []
+    for _ in range(steps):
+        if flush is not None:
+            flush.zero_()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        fn()
+        b.record()
+        b.synchronize()
+        ts.append(a.elapsed_time(b))
+    return ts
+
+
+def bound_and_frac(ops: float, nbytes: float, ms: float, tensor_peak: float, hbm_gbs: float):
+    """The roof that bounds a launch (the slower of ops / tensor peak and bytes / HBM peak) and the fraction of it
+    reached: floor time / measured time."""
+    t_tensor = ops / (tensor_peak * 1e12) * 1e3
+    t_hbm = nbytes / (hbm_gbs * 1e9) * 1e3
+    bound = "tensor" if t_tensor >= t_hbm else "hbm"
+    return bound, max(t_tensor, t_hbm) / ms
+
+
+def other_configs(tensor_peak: float, hbm_gbs: float, steps: int = 20, warmup: int = 5):
+    """The other benchmark workloads (single 3x3 layer, GEMM sweep int32 + fused, stem / down-sampling layers, block
+    stack), AUTO engine, 20 launches each with L2 flushed in between: median and min time, TOP/s and the fraction of
+    the bounding roof (tensor pipe or HBM, on algorithmic bytes: packed inputs + weights + output)."""
+    import torch
+    from paper_2010_00704_b200 import binding
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    rng = np.random.default_rng(synth.seed_for(2, 77))
+    rows = []
+
+    def add(name, fn, ops, nbytes):
+        ts = timed_launches(fn, steps, warmup, flush)
+        med, mn = float(np.median(ts)), float(min(ts))
+        bound, frac = bound_and_frac(ops, nbytes, med, tensor_peak, hbm_gbs)
+        rows.append({"name": name, "ms_median": med, "ms_min": mn, "tops": ops / (med / 1e3) / 1e12, "bound": bound,
+                     "frac": frac, "algorithmic_bytes": int(nbytes)})
+
+    def conv_case(tag, l, B, fused=True):
+        x = torch.from_numpy(synth.random_bits(rng, (l.in_bytes(B),))).cuda()
+        Wb = torch.from_numpy(synth.random_bits(rng, (l.w_bytes(),))).cuda()
+        if fused:
+            thr = torch.from_numpy(synth.thresholds(rng, l.K, l.C_out)).cuda()
+            out = torch.empty(l.out_bits_bytes(B), dtype=torch.uint8, device="cuda")
+            fn = lambda: binding.bcnn_conv2d_b1_fused(x, Wb, thr, out, B, l.H, l.W, l.C_in, l.C_out, l.k, l.k, l.stride, l.pad)
+            ob = l.out_bits_bytes(B)
+        else:
+            out = torch.empty(l.M(B) * l.C_out, dtype=torch.int32, device="cuda")
+            fn = lambda: binding.bcnn_conv2d_b1(x, Wb, out, B, l.H, l.W, l.C_in, l.C_out, l.k, l.k, l.stride, l.pad)
+            ob = 4 * l.M(B) * l.C_out
+        add(f"{tag} {l.name} B={B} M={l.M(B)} N={l.C_out} K={l.K} {'fused' if fused else 'int32'}", fn, l.ops(B),
+            l.in_bytes(B) + l.w_bytes() + ob)
+
+    conv_case("single3x3:", wl.SINGLE_3X3, wl.SINGLE_3X3_BATCH, fused=False)
+    for mn_ in wl.GEMM_SWEEP_MN:
+        for k in wl.GEMM_SWEEP_K:
+            M = N = mn_
+            A = torch.from_numpy(synth.random_bits(rng, (M, k // 8))).cuda()
+            Wb = torch.from_numpy(synth.random_bits(rng, (N, k // 8))).cuda()
+            thr = torch.from_numpy(synth.thresholds(rng, k, N)).cuda()
+            out32 = torch.empty(M * N, dtype=torch.int32, device="cuda")
+            outb = torch.empty(M * N // 8, dtype=torch.uint8, device="cuda")
+            ops = wl.gemm_ops(M, N, k)
+            add(f"gemm M=N={M} K={k} int32", lambda: binding.bcnn_gemm_b1(A, Wb, out32, M, N, k), ops, (M + N) * k // 8 + 4 * M * N)
+            add(f"gemm M=N={M} K={k} fused", lambda: binding.bcnn_gemm_b1_fused(A, Wb, thr, outb, M, N, k), ops,
+                (M + N) * k // 8 + M * N // 8)
+            del A, Wb, thr, out32, outb
+    for l in wl.STEM_DOWN:
+        conv_case("stem/down:", l, wl.STEM_DOWN_BATCH)
+    for l in wl.BLOCK_STACK:
+        conv_case("block stack:", l, wl.BLOCK_STACK_BATCH)
+    return rows
+
 
 def run_gpu(args):
     import torch
@@ -221,6 +383,7 @@ def run_gpu(args):
     build.build()
     binding.load()
     peaks = load_peaks()
+    probes = run_probes() if rank == 0 else None
 
     layers = wl.BACKBONE18
     B = wl.BACKBONE18_BATCH
@@ -237,7 +400,8 @@ def run_gpu(args):
             dist.barrier()
         torch.cuda.synchronize()
 
-    # ---- device-resident timed region (CUDA graph replay of pack + 18 layers)
+    # ---- device-resident timed region (CUDA graph replay of the fused stem + 17 layers); an event after every
+    # step gives the per-step times too
     chain.capture()
     for _ in range(max(args.warmup, 3)):
         chain.run()
@@ -246,26 +410,43 @@ def run_gpu(args):
     if rank == 0:
         sampler.start()
         time.sleep(0.3)
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    marks = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
     barrier()
-    e0.record()
-    for _ in range(args.steps):
+    marks[0].record()
+    for s in range(args.steps):
         chain.run()
-    e1.record()
+        marks[s + 1].record()
     barrier()
-    ms_total = reduce_max(e0.elapsed_time(e1), device)
+    ms_total = reduce_max(marks[0].elapsed_time(marks[-1]), device)
+    step_ms = [marks[s].elapsed_time(marks[s + 1]) for s in range(args.steps)]
     clocks = sampler.stop() if rank == 0 else None
     err = binding.bcnn_device_error()
     if err != 0:
-        raise SystemExit(f"device-side error code {err}")
+        raise SystemExit(f"device-side error code {err}: {binding.status_string(err)}")
     ms_step = ms_total / args.steps
     value = aggregate_throughput(ops_step * args.steps, world, ms_total / 1e3) / 1e12
+
+    # ---- sustained leg: the same graph replayed back to back for at least two seconds (warm, power-limited GPU)
+    n_sus = max(args.steps, int(np.ceil(args.sustain_seconds * 1e3 / ms_step)))
+    sampler_s = ClockSampler(local_rank)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    if rank == 0:
+        sampler_s.start()
+    e0.record()
+    for _ in range(n_sus):
+        chain.run()
+    e1.record()
+    barrier()
+    ms_sus = reduce_max(e0.elapsed_time(e1), device)
+    clocks_sus = sampler_s.stop() if rank == 0 else None
+    value_sus = aggregate_throughput(ops_step * n_sus, world, ms_sus / 1e3) / 1e12
 
     # ---- end to end: pinned host input -> device, whole path, result back to the host
     out_host = torch.empty(chain.outs[-1].numel(), dtype=torch.uint8).pin_memory()
     def e2e_step():
         # host -> device copy of this step's input (copy stream, overlapping the previous step's kernels),
-        # pack + 18 layers, packed result back to the host
+        # fused stem + 17 layers, packed result back to the host
         chain.run_from_host(x_host, out_host)
     for _ in range(3):
         e2e_step()
@@ -278,12 +459,15 @@ def run_gpu(args):
     ms_e2e = reduce_max(e0.elapsed_time(e1), device)
     e2e_value = aggregate_throughput(ops_step * args.steps, world, ms_e2e / 1e3) / 1e12
 
-    # ---- per-kernel pass: the same launches, one CUDA-event pair around each
+    # ---- per-kernel pass: the same launches, one CUDA-event pair around each; clocks sampled during it
     nl = len(layers)
     per = np.zeros((args.steps, nl + 1))
     evs = [[(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(nl + 1)]
            for _ in range(args.steps)]
     fused_stem = chain.fuse_stem
+    sampler_k = ClockSampler(local_rank)
+    if rank == 0:
+        sampler_k.start()
     for s in range(args.steps):
         a, b = evs[s][0]
         a.record()
@@ -300,31 +484,53 @@ def run_gpu(args):
             b.record()
             cur = o
     torch.cuda.synchronize()
+    clocks_k = sampler_k.stop() if rank == 0 else None
     for s in range(args.steps):
         for i in range(nl + 1):
             if not (i == 1 and fused_stem):
                 per[s, i] = evs[s][i][0].elapsed_time(evs[s][i][1])
     per_ms = per.mean(axis=0)
-    # dense 8-bit integer tensor peak = measured bf16 peak x the nominal 2:1 ratio (4.5 : 2.25 PFLOP/s);
-    # the sustained figure, because the kernels are timed inside a long step
-    tensor_peak = 2.0 * peaks["bf16_tflops_sustained"]
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return 0
+
+    # Tensor peak: the tcgen05.mma kind::i8 rate measured in this process by the tensor-memory-resident probe
+    # (N = 256 instructions back to back).  Beside it, 2 x the measured bf16 GEMM peaks (the nominal 2:1 ratio of
+    # the dense 8-bit and 16-bit pipes): burst for launches timed alone at the maximum clock, sustained for a warm,
+    # power-limited GPU.  Which of the two applies to the per-launch times is decided by the clocks sampled
+    # while those launches ran.
+    tensor_peak = probes["tcgen05_i8_n256"]
+    peak_alt = {"2x_bf16_burst": 2.0 * peaks["bf16_tflops"], "2x_bf16_sustained": 2.0 * peaks["bf16_tflops_sustained"]}
+    def regime_of(c):
+        if not c or not c.get("sm_mhz") or not c.get("sm_max_mhz"):
+            return "unknown"
+        return "burst" if c["sm_mhz"] >= 0.95 * c["sm_max_mhz"] else "sustained"
+    regime = regime_of(clocks_k)
+    alt_key = "2x_bf16_sustained" if regime == "sustained" else "2x_bf16_burst"
     engines = [binding.bcnn_auto_engine(B, l.H, l.W, l.C_in, l.C_out, l.k, l.k, l.stride, l.pad) for l in layers]
     if fused_stem:
         engines[0] = "stem"                       # the first layer runs inside the stem kernel (slot 0 of per_ms)
     kernel_of = {"tc_i8": "conv_tc_i8_kernel (tcgen05 kind::i8)", "mma_s8": "conv_mma_s8_kernel (mma.sync u8)",
                  "mma_b1": "conv_mma_b1_kernel (mma.sync b1)",
-                 "tc_ws": "conv_tc_ws_kernel (tcgen05 kind::i8, weights resident in shared memory)", "lop3": "conv_k32_kernel (CUDA-core xor + popc)"}
+                 "tc_ws": "conv_tc_ws_kernel (tcgen05 kind::i8, weights resident in shared memory)",
+                 "tc_pw": "conv_tc_pw_kernel (tcgen05 kind::i8, pointwise layers, bulk-copied rows)",
+                 "lop3": "conv_k32_kernel (CUDA-core xor + popc)"}
     lay_ms = [float(per_ms[0]) if engines[i] == "stem" else float(per_ms[i + 1]) for i in range(nl)]
-    per_layer = [{"layer": l.name + (" (with the pack, one kernel)" if engines[i] == "stem" else ""), "engine": engines[i],
-                  "ms": lay_ms[i], "tops": l.ops(B) / (lay_ms[i] / 1e3) / 1e12} for i, l in enumerate(layers)]
+    per_layer = []
+    for i, l in enumerate(layers):
+        nbytes = l.in_bytes(B) + l.w_bytes() + l.out_bits_bytes(B)
+        bound, frac = bound_and_frac(l.ops(B), nbytes, lay_ms[i], tensor_peak, peaks["hbm_gbs"])
+        per_layer.append({"layer": l.name + (" (with the pack, one kernel)" if engines[i] == "stem" else ""), "engine": engines[i],
+                          "ms": lay_ms[i], "tops": l.ops(B) / (lay_ms[i] / 1e3) / 1e12, "bound": bound, "frac": frac})
     groups = []
     for en in sorted(set(engines) - {"stem"}):
         idx = [i for i, e in enumerate(engines) if e == en]
         g_ms = float(sum(per_ms[i + 1] for i in idx))
         g_ops = float(sum(layers[i].ops(B) for i in idx))
-        # the CUDA-core kernel sits on the population-count unit: its peak is the xor + popc rate that
-        # tools/engine_peaks measures register-resident (385 TOP/s at 1965 MHz)
-        g_bound, g_peak = ("alu", POPC_PEAK_TOPS) if en == "lop3" else ("tensor", tensor_peak)
+        # the CUDA-core kernel sits on the population-count unit: its peak is the xor + popc rate of the probe
+        g_bound, g_peak = ("alu", probes["xor_popc"]) if en == "lop3" else ("tensor", tensor_peak)
         groups.append({"kernel": kernel_of[en], "launches_per_step": len(idx), "ms_per_step": g_ms,
                        "share_of_step": g_ms / float(per_ms.sum()), "bound": g_bound,
                        "achieved": g_ops / (g_ms / 1e3) / 1e12, "peak": g_peak, "unit": "TOP/s",
@@ -336,13 +542,24 @@ def run_gpu(args):
     top = max((i for i, e in enumerate(engines) if e == dom_engine), key=lambda i: per_ms[i + 1])
     lt = layers[top]
     top_tops = lt.ops(B) / (per_ms[top + 1] / 1e3) / 1e12
+    src_of = {"tc_ws": ["conv_tc_ws.cu", "tc_common.cuh"], "tc_i8": ["conv_tc_i8.cu", "tc_common.cuh"],
+              "tc_pw": ["conv_tc_pw.cu", "tc_common.cuh"]}
     roofline = {
         "kernel": groups[0]["kernel"], "launch": f"{lt.name}: M={lt.M(B)} N={lt.C_out} K={lt.K}",
         "bound": "tensor", "achieved": top_tops, "peak": tensor_peak, "unit": "TOP/s", "frac": top_tops / tensor_peak,
-        "peak_source": f"2 x sustained bf16 GEMM of the {peaks['source']} peaks (dense 8-bit tensor pipe), of {peaks['source']}",
+        "peak_source": "tcgen05.mma kind::i8 (M=128, N=256, K=32, A in tensor memory) issued back to back, measured in this "
+                       f"process by bench_probes.cu; peak_alt = 2 x the {peaks['source']} bf16 GEMM peaks (MEASURED_PEAKS.json), "
+                       f"of {peaks['source']}",
+        "peak_alt": peak_alt, "frac_alt": {k: top_tops / v for k, v in peak_alt.items()},
+        "regime": regime, "frac_of_regime_peak": top_tops / peak_alt[alt_key],
+        "regime_source": "median SM clock sampled while the per-launch events ran: burst when within 5 % of the maximum",
+        "clocks_during_launch_timing": clocks_k,
         "launch_ms": float(per_ms[top + 1]),
-        "traffic": ROOFLINE_TRAFFIC.get(lt.name),
+        "launch_ms_x_sm_mhz": (float(per_ms[top + 1]) * clocks_k["sm_mhz"]) if clocks_k and clocks_k.get("sm_mhz") else None,
+        "ops_per_launch": int(lt.ops(B)),
+        "traffic": roofline_traffic(f"conv_{dom_engine}_{lt.name}.txt", src_of.get(dom_engine, [])),
         "kernels": groups,
+        "instruction_peaks_tops": probes,
     }
     # pack: 16 bytes read, 4 written per pixel; the fused stem writes the first layer's 4 bytes instead
     pack_bytes = B * H * W * C * 4 + B * H * W * (layers[0].C_out if fused_stem else C * R) // 8
@@ -351,21 +568,24 @@ def run_gpu(args):
             "achieved": pack_bytes / (per_ms[0] / 1e3) / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s",
             "frac": pack_bytes / (per_ms[0] / 1e3) / 1e9 / peaks["hbm_gbs"], "algorithmic_bytes": pack_bytes}
 
-    if rank != 0:
-        if world > 1:
-            dist.destroy_process_group()
-        return 0
-
+    configs = other_configs(tensor_peak, peaks["hbm_gbs"]) if world == 1 and not args.no_configs else None
+    err = binding.bcnn_device_error()
+    if err != 0:
+        raise SystemExit(f"device-side error code {err}: {binding.status_string(err)}")
     cpu = cpu_baseline() if world == 1 and not args.no_cpu_baseline else None
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-        "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+        "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "ms_per_step_median": float(np.median(step_ms)),
+        "ms_per_step_min": float(min(step_ms)), "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": "b1 (sign bits) with int32 accumulation", "data": "synthetic",
         "config": {"workload": WORKLOAD, "batch_per_gpu": B, "layers": nl,
                    "cache": "inputs larger than L2 (205.5 MB fp32 input read every step)",
                    "launch": f"CUDA graph replay of {chain.launches_per_run} kernels"},
         "images_per_s": B * world * args.steps / (ms_total / 1e3),
         "clocks": clocks,
+        "value_sustained": value_sus,
+        "sustained": {"value": value_sus, "unit": UNIT, "steps": n_sus, "seconds": ms_sus / 1e3, "ms_per_step": ms_sus / n_sus,
+                      "images_per_s": B * world * n_sus / (ms_sus / 1e3), "clocks": clocks_sus, "regime": regime_of(clocks_sus)},
         "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": int(x_host.numel() * 4),
                 "d2h_bytes_per_step": int(out_host.numel()), "ms_per_step": ms_e2e / args.steps,
                 "api": "FusedChain.run_from_host: pinned host input, copy stream overlapping the previous step",
@@ -374,6 +594,7 @@ def run_gpu(args):
         "roofline": roofline,
         "pack": pack,
         "per_layer": per_layer,
+        "configs": configs,
         "cpu_baseline": cpu,
     }
     print(json.dumps(line))
@@ -585,6 +806,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-configs", action="store_true", help="skip the other workloads (single layer, GEMM sweep, stem / down, block stack)")
+    ap.add_argument("--sustain-seconds", type=float, default=2.0, help="length of the sustained leg")
     ap.add_argument("--batch", type=int, default=256, help="paper1x1 mode: images per step")
     ap.add_argument("--epilogue", default="threshold", choices=["threshold", "module"],
                     help="paper1x1 mode: integer threshold, or the full convolution module (batch norm, fp16 identity, PReLU, next sign)")

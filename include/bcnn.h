@@ -45,7 +45,10 @@ typedef enum bcnn_status {
     BCNN_ERR_INVALID_ARG = -1, /* null pointer, non-positive size, empty output */
     BCNN_ERR_UNSUPPORTED = -2, /* channel count not a multiple of 32, size limits */
     BCNN_ERR_ALIGNMENT = -3,   /* a data pointer is not 16-byte aligned */
-    BCNN_ERR_CUDA = -4         /* the CUDA runtime refused a launch */
+    BCNN_ERR_CUDA = -4,        /* the CUDA runtime refused a launch */
+    BCNN_ERR_WORKSPACE = -5,   /* a caller-provided scratch buffer is too small (no call takes one today:
+                                  bcnn_workspace_bytes() is 0 for every shape; the value is reserved) */
+    BCNN_ERR_TIMEOUT = -6      /* a bounded device-side wait gave up (see bcnn_device_status) */
 } bcnn_status;
 
 /* Engines of the inner product; BCNN_ENGINE_AUTO picks per shape. */
@@ -169,12 +172,40 @@ int bcnn_gemm_b1_engine(int engine, const void *A_bits, const void *W_bits, cons
 int bcnn_auto_engine(int B, int H, int W, int C_in, int C_out, int kh, int kw, int stride, int pad, int fused);
 
 /*
+ * Scratch memory (global memory beyond the inputs and outputs) a convolution of this shape needs, in bytes
+ * (fused != 0: the packed output).  Every kernel of the library works out of its inputs, outputs, shared and
+ * tensor memory, so this is 0 for every valid shape and no call takes a workspace argument; an invalid shape
+ * also gives 0 (the call itself reports the error).  A GEMM is the shape (1, M, 1, K, N, 1, 1, 1, 0).
+ */
+size_t bcnn_workspace_bytes(int B, int H, int W, int C_in, int C_out, int kh, int kw, int stride, int pad, int fused);
+
+/*
  * Device-side error word.  Kernels that wait on hardware barriers give up after a
  * bounded number of polls and record a non-zero code here instead of hanging.
  * Reads the word of the current device (synchronises that device) and clears it.
- * Returns the code (0 = no error) or a negative bcnn_status.
+ * Returns the code (0 = no error) or a negative bcnn_status.  bcnn_status_string names the codes
+ * (which engine, which of its roles gave up).
  */
 int bcnn_device_error(void);
+
+/*
+ * The same check as a status: synchronises the current device, reads and clears the error word and returns
+ * BCNN_OK, BCNN_ERR_TIMEOUT when a bounded wait had given up (the results of the calls since the last check
+ * are then undefined; the context stays usable), or BCNN_ERR_CUDA.  *code, when not NULL, receives the raw
+ * code (0 = none).
+ */
+int bcnn_device_status(int *code);
+
+/*
+ * Self-test of the bounded waits: launches one small kernel that allocates tensor memory and lets one warp
+ * wait, with the library's wait helper and a limit of `polls` polls (1 <= polls <= 65536), on a barrier that
+ * nothing ever arrives on.  The wait gives up, raises the CTA's abort flag (which the other warps of the CTA,
+ * parked on a second barrier, notice), records BCNN_SELFTEST_TIMEOUT_CODE in the device error word, the kernel
+ * frees its tensor memory and ends normally.  Enqueues only; bcnn_device_error() / bcnn_device_status() then
+ * report the code.  Nothing else in the library calls it.
+ */
+#define BCNN_SELFTEST_TIMEOUT_CODE 120
+int bcnn_selftest_wait_timeout(int polls, void *stream);
 
 const char *bcnn_status_string(int status);
 int bcnn_version(void);

@@ -21,9 +21,13 @@ ENGINES = {"auto": ENGINE_AUTO, "lop3": ENGINE_LOP3, "mma_b1": ENGINE_MMA_B1, "t
 
 EXPORTS = (
     "bcnn_pack", "bcnn_stem_fused", "bcnn_gemm_b1", "bcnn_gemm_b1_fused", "bcnn_conv2d_b1", "bcnn_conv2d_b1_fused", "bcnn_conv2d_b1_module",
-    "bcnn_conv2d_b1_engine", "bcnn_gemm_b1_engine", "bcnn_auto_engine", "bcnn_device_error", "bcnn_status_string",
-    "bcnn_version",
+    "bcnn_conv2d_b1_engine", "bcnn_gemm_b1_engine", "bcnn_auto_engine", "bcnn_device_error", "bcnn_device_status",
+    "bcnn_workspace_bytes", "bcnn_selftest_wait_timeout", "bcnn_status_string", "bcnn_version",
 )
+
+# bcnn_status values
+OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_ALIGNMENT, ERR_CUDA, ERR_WORKSPACE, ERR_TIMEOUT = 0, -1, -2, -3, -4, -5, -6
+SELFTEST_TIMEOUT_CODE = 120
 
 _lib = None
 
@@ -53,10 +57,14 @@ def load() -> ctypes.CDLL:
         lib.bcnn_gemm_b1_engine.argtypes = [i32, vp, vp, vp, vp, i64, i32, i32, vp]
         lib.bcnn_auto_engine.argtypes = [i32] * 10
         lib.bcnn_device_error.argtypes = []
+        lib.bcnn_device_status.argtypes = [ctypes.POINTER(ctypes.c_int)]
+        lib.bcnn_workspace_bytes.argtypes = [i32] * 10
+        lib.bcnn_workspace_bytes.restype = ctypes.c_size_t
+        lib.bcnn_selftest_wait_timeout.argtypes = [i32, vp]
         lib.bcnn_status_string.argtypes = [i32]
         lib.bcnn_status_string.restype = ctypes.c_char_p
         for name in EXPORTS:
-            if name != "bcnn_status_string":
+            if name not in ("bcnn_status_string", "bcnn_workspace_bytes"):
                 getattr(lib, name).restype = i32
         _lib = lib
     return _lib
@@ -150,3 +158,19 @@ def bcnn_auto_engine(B, H, W, C_in, C_out, kh, kw, stride, pad, fused=True) -> s
 
 def bcnn_device_error() -> int:
     return load().bcnn_device_error()
+
+
+def bcnn_device_status():
+    """(status, code): BCNN_OK / BCNN_ERR_TIMEOUT / BCNN_ERR_CUDA and the raw device error code."""
+    code = ctypes.c_int(0)
+    st = load().bcnn_device_status(ctypes.byref(code))
+    return st, code.value
+
+
+def bcnn_workspace_bytes(B, H, W, C_in, C_out, kh, kw, stride, pad, fused=True) -> int:
+    return int(load().bcnn_workspace_bytes(B, H, W, C_in, C_out, kh, kw, stride, pad, 1 if fused else 0))
+
+
+def bcnn_selftest_wait_timeout(polls: int = 256):
+    """Enqueue the self-test kernel whose bounded wait runs out (see include/bcnn.h)."""
+    _check(load().bcnn_selftest_wait_timeout(int(polls), _stream()), "bcnn_selftest_wait_timeout")

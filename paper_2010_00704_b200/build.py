@@ -52,17 +52,5 @@ def build(force: bool = False, verbose: bool = False) -> str:
     return LIB
 
 
-def build_tools() -> str:
-    """Compile the stand-alone instruction-throughput probe (tools/engine_peaks.cu)."""
-    src = os.path.join(PKG, "tools", "engine_peaks.cu")
-    exe = os.path.join(PKG, "tools", "engine_peaks")
-    if not os.path.exists(exe) or os.path.getmtime(exe) < os.path.getmtime(src):
-        subprocess.run([os.environ.get("NVCC", "nvcc"), "-gencode", "arch=compute_100a,code=sm_100a", "-O3",
-                        "-o", exe, src], check=True)
-    return exe
-
-
 if __name__ == "__main__":
     print(build(force="--force" in sys.argv, verbose="-v" in sys.argv))
-    if "--tools" in sys.argv:
-        print(build_tools())

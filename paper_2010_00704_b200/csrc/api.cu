@@ -255,6 +255,27 @@ int bcnn_device_error(void)
     return v;
 }
 
+int bcnn_device_status(int *code)
+{
+    const int v = bcnn_device_error();
+    if (code) *code = v > 0 ? v : 0;
+    if (v < 0) return v;
+    return v == 0 ? BCNN_OK : BCNN_ERR_TIMEOUT;
+}
+
+size_t bcnn_workspace_bytes(int B, int H, int W, int C_in, int C_out, int kh, int kw, int stride, int pad, int fused)
+{
+    // no kernel uses global memory beyond its inputs and outputs, whatever the shape
+    (void)B; (void)H; (void)W; (void)C_in; (void)C_out; (void)kh; (void)kw; (void)stride; (void)pad; (void)fused;
+    return 0;
+}
+
+int bcnn_selftest_wait_timeout(int polls, void *stream)
+{
+    if (polls < 1 || polls > 65536) return BCNN_ERR_INVALID_ARG;
+    return launch_selftest_wait_timeout(polls, static_cast<cudaStream_t>(stream));
+}
+
 const char *bcnn_status_string(int status)
 {
     switch (status) {
@@ -263,6 +284,16 @@ const char *bcnn_status_string(int status)
     case BCNN_ERR_UNSUPPORTED: return "unsupported shape or engine";
     case BCNN_ERR_ALIGNMENT: return "pointer not 16-byte aligned";
     case BCNN_ERR_CUDA: return "CUDA runtime error";
+    case BCNN_ERR_WORKSPACE: return "workspace too small";
+    case BCNN_ERR_TIMEOUT: return "a bounded device-side wait gave up";
+    // device error word: which bounded wait gave up
+    case 101: return "device wait timed out: streaming tcgen05 engine, producer waiting for a free ring slot";
+    case 102: return "device wait timed out: streaming tcgen05 engine, control warp waiting for a full slot or a free accumulator";
+    case 103: return "device wait timed out: streaming tcgen05 engine, epilogue waiting for an accumulator";
+    case 111: return "device wait timed out: weight-stationary tcgen05 engine, producer waiting for a free ring slot";
+    case 112: return "device wait timed out: weight-stationary tcgen05 engine, control warp waiting for a full slot or a free accumulator";
+    case 113: return "device wait timed out: weight-stationary tcgen05 engine, epilogue waiting for an accumulator";
+    case BCNN_SELFTEST_TIMEOUT_CODE: return "device wait timed out: self-test (expected)";
     default: return status > 0 ? "device-side error code" : "unknown status";
     }
 }

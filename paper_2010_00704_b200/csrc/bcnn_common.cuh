@@ -79,6 +79,7 @@ int launch_conv_tc_ws(const ConvProblem &p, cudaStream_t stream);
 bool conv_tc_ws_supports(const ConvProblem &p);
 int launch_conv_tc_i8(const ConvProblem &p, cudaStream_t stream);
 bool conv_tc_i8_supports(const ConvProblem &p);
+int launch_selftest_wait_timeout(int polls, cudaStream_t stream);
 int *device_error_word();   // device address of the error word of the current device (nullptr on failure)
 
 }  // namespace bcnn

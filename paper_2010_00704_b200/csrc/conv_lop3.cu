@@ -227,7 +227,7 @@ bool conv_lop3_pointwise_k32(const ConvProblem &p)
 int launch_conv_lop3(const ConvProblem &p, cudaStream_t stream)
 {
     if (conv_lop3_pointwise_k32(p)) return p.thr ? launch_k32<true>(p, stream) : launch_k32<false>(p, stream);
-    dim3 grid((p.M + BM - 1) / BM, (p.C_out + BN - 1) / BN);
+    dim3 grid((unsigned)(((long)p.M + BM - 1) / BM), (p.C_out + BN - 1) / BN);
     if (grid.y > 65535) return BCNN_ERR_UNSUPPORTED;
     if (p.thr)
         conv_lop3_kernel<true><<<grid, 256, 0, stream>>>(p);

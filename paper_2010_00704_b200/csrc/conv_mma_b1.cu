@@ -272,7 +272,7 @@ int launch_variant(const ConvProblem &p, cudaStream_t stream)
 {
     constexpr int BN = 32 * WN;
     const int smem = STAGES * (BM + BN) * ROW_BYTES;
-    dim3 grid((p.M + BM - 1) / BM, (p.C_out + BN - 1) / BN);
+    dim3 grid((unsigned)(((long)p.M + BM - 1) / BM), (p.C_out + BN - 1) / BN);
     if (grid.y > 65535) return BCNN_ERR_UNSUPPORTED;
     cudaError_t e;
     if (p.thr) {

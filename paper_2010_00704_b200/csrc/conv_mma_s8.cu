@@ -73,7 +73,9 @@ conv_mma_s8_kernel(const ConvProblem p)
         // with acc = 128 * popc(A and G) and pa = popc(A):
         //   int32:  value = (acc >> 5) - 2*pa + (K - 2*pop)
         //   fused:  bit   = acc - 64*pa - 32*(thr - K + 2*pop) >= 0
-        colc[c] = FUSED ? -32 * ((n < p.C_out ? __ldg(p.thr + n) : 0) - p.K + 2 * pop) : p.K - 2 * pop;
+        // (a threshold beyond +-(K + 1) decides like that bound; clamping keeps the constant inside int32)
+        const int thr_n = max(min(FUSED && n < p.C_out ? __ldg(p.thr + n) : 0, p.K + 1), -p.K - 1);
+        colc[c] = FUSED ? -32 * (thr_n - p.K + 2 * pop) : p.K - 2 * pop;
     }
     for (int tp = tid; tp < ntaps; tp += THREADS) tapoff[tp] = ((tp / p.kw) * p.W + (tp % p.kw)) * p.cw;
     __syncthreads();

@@ -84,7 +84,7 @@ conv_tc_i8_kernel(const ConvProblem p, const int ktab_words)
     const int tid = threadIdx.x;
     const int warp = tid >> 5, lane = tid & 31;
     const int ktiles = (p.kwords + 3) >> 2;
-    const int m_tiles = (p.M + BM - 1) / BM;
+    const int m_tiles = (p.M - 1) / BM + 1;                  // M >= 1; no overflow for M close to 2^31
     const int n_tiles = (p.C_out + BN - 1) / BN;
     const int total_tiles = m_tiles * n_tiles;
     const int my_tiles = ((int)blockIdx.x < total_tiles) ? (total_tiles - 1 - (int)blockIdx.x) / (int)gridDim.x + 1 : 0;
@@ -447,7 +447,8 @@ conv_tc_i8_kernel(const ConvProblem p, const int ktab_words)
                 if (!is_a && first_group) {
                     const int tile = (int)blockIdx.x + c_ti * (int)gridDim.x;
                     const int n = (tile / m_tiles) * BN + row;
-                    const int thr_n = (FUSED && n < p.C_out) ? __ldg(p.thr + n) : 0;
+                    // (a threshold beyond +-(K + 1) decides like that bound; clamping keeps the constant inside int32)
+                    const int thr_n = max(min((FUSED && n < p.C_out) ? __ldg(p.thr + n) : 0, p.K + 1), -p.K - 1);
                     cst += FUSED ? -32 * (thr_n - p.K) : p.K;
                 }
                 const uint32_t part = consts + (uint32_t)(((c_ti % SLOTS) * C::SLOT_INTS + grp * (BM + BN) + crow) * 4);

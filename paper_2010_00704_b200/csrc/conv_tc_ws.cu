@@ -118,7 +118,7 @@ conv_tc_ws_kernel(const ConvProblem p)
     const WsLayout L = ws_layout<BN, G, DUAL, TEAMS>(p.kwords, MODE);
     const int ktiles = L.ktiles;
     constexpr int STAGES = C::STAGES;
-    const int m_tiles = (p.M + BM - 1) / BM;
+    const int m_tiles = (p.M - 1) / BM + 1;                  // M >= 1; no overflow for M close to 2^31
     // N slices: a CTA keeps the weights of one slice of BN output channels and walks row tiles mb, mb + mstride, ...
     // (the grid is a multiple of the slice count)
     const int n_tiles = (p.C_out + BN - 1) / BN;
@@ -159,7 +159,7 @@ conv_tc_ws_kernel(const ConvProblem p)
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
 
-    // ---- one-off: expand the weight tile (+ the all-ones row), column constants, K-word table
+    // ---- one-off: expand the weight tile, per-channel constants, K-word table
     for (int idx = tid; idx < ktiles * BN; idx += C::THREADS) {
         const int kt = idx / BN, row = idx - kt * BN;
         const uint32_t row_addr = wexp + (uint32_t)kt * C::W_TILE_BYTES + (uint32_t)row * ROWB;

@@ -38,9 +38,10 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
 // Bounded wait with back-off.  A polling warp competes with the MMA-issuing warp for issue
 // slots, so after a first failed poll the waiter sleeps between polls.  The polling loop is kept
 // out of line: the common case is one successful try_wait.
-static __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *err, int code)
+static __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *err, int code,
+                                                   uint32_t limit = WAIT_LIMIT)
 {
-    for (uint32_t it = 0; it < WAIT_LIMIT; ++it) {
+    for (uint32_t it = 0; it < limit; ++it) {
         __nanosleep(SLEEP_NS);
         if (mbar_try_wait(bar, parity)) return true;
         if ((it & 255u) == 255u && *abort_flag) return false;
@@ -49,17 +50,19 @@ static __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity
     if (err) atomicCAS(err, 0, code);
     return false;
 }
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *err, int code)
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *err, int code,
+                                          uint32_t limit = WAIT_LIMIT)
 {
     if (mbar_try_wait(bar, parity)) return true;
-    return mbar_wait_slow(bar, parity, abort_flag, err, code);
+    return mbar_wait_slow(bar, parity, abort_flag, err, code, limit);
 }
 // Whole-warp wait: one try_wait per lane and a vote in the common case.
-__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *err, int code)
+__device__ __forceinline__ bool mbar_wait_warp(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *err, int code,
+                                               uint32_t limit = WAIT_LIMIT)
 {
     bool ok = mbar_try_wait(bar, parity);
     if (__all_sync(0xffffffffu, ok)) return true;
-    if (!ok) ok = mbar_wait_slow(bar, parity, abort_flag, err, code);
+    if (!ok) ok = mbar_wait_slow(bar, parity, abort_flag, err, code, limit);
     return __all_sync(0xffffffffu, ok);
 }
 __device__ __forceinline__ void mbar_arrive_pred(uint32_t bar, uint32_t pred)

@@ -28,6 +28,23 @@ def test_status_strings_and_version():
     assert binding.version() >= 100
     assert binding.status_string(0) == "ok"
     assert "align" in binding.status_string(-3)
+    assert "workspace" in binding.status_string(binding.ERR_WORKSPACE)
+    assert "wait" in binding.status_string(binding.ERR_TIMEOUT)
+    # the device error codes name the engine and the role whose wait gave up
+    for code in (101, 102, 103, 111, 112, 113, binding.SELFTEST_TIMEOUT_CODE):
+        assert "timed out" in binding.status_string(code)
+    assert binding.status_string(77) == "device-side error code"
+
+
+def test_workspace_bytes_is_zero_for_every_shape():
+    # no kernel uses scratch memory: the query exists so that callers can size one buffer per model anyway
+    from paper_2010_00704_b200 import build, binding, workloads as wl
+    build.build()
+    for l in wl.BACKBONE18 + wl.BLOCK_STACK + wl.STEM_DOWN:
+        for fused in (False, True):
+            assert binding.bcnn_workspace_bytes(256, l.H, l.W, l.C_in, l.C_out, l.k, l.k, l.stride, l.pad, fused) == 0
+    assert binding.bcnn_workspace_bytes(1, 16384, 1, 9216, 16384, 1, 1, 1, 0) == 0      # a GEMM of the sweep
+    assert binding.bcnn_workspace_bytes(1, 4, 4, 48, 32, 1, 1, 1, 0) == 0                # invalid shape: still 0
 
 
 def test_argument_validation_needs_no_device():
@@ -48,3 +65,5 @@ def test_argument_validation_needs_no_device():
     assert lib.bcnn_pack(a, None, a, 1, 2, 2, 12, 2, None) == -2
     assert lib.bcnn_pack(None, None, a, 1, 2, 2, 32, 1, None) == -1
     assert lib.bcnn_conv2d_b1_engine(99, a, a, None, a, 1, 4, 4, 32, 8, 3, 3, 1, 1, None) == -2
+    assert lib.bcnn_selftest_wait_timeout(0, None) == -1
+    assert lib.bcnn_selftest_wait_timeout(1 << 20, None) == -1

@@ -85,6 +85,16 @@ CONV_SHAPES = [
 ]
 
 
+def plant_extreme_thresholds(thr, K):
+    """Thresholds at and beyond the reachable sums, up to the ends of int32 (a batch norm whose scale vanishes
+    folds to an unbounded threshold: INT_MAX = the channel never fires, INT_MIN = it always does)."""
+    ext = np.array([-2**31, 2**31 - 1, -K - 2, -K - 1, -K, K, K + 1, K + 2, 2**26, -2**26, 2**30, -2**30,
+                    2**26 + K, -(2**26) - K, 2**31 - 1 - K, -2**31 + K], dtype=np.int64).astype(np.int32)
+    n = min(len(ext), max(1, len(thr) // 2))
+    thr[1:2 * n:2] = ext[:n]                      # odd channels (the even ones keep ties / uniform draws)
+    return thr
+
+
 @pytest.mark.parametrize("engine", ENGINES)
 @pytest.mark.parametrize("shape", CONV_SHAPES)
 def test_conv_int32_and_fused(bk, oracle, shape, engine):
@@ -98,6 +108,9 @@ def test_conv_int32_and_fused(bk, oracle, shape, engine):
     K = kh * kw * Ci
     thr = synth.thresholds(rng, K, Co)
     thr[::3] = want.reshape(-1, Co)[0, ::3]           # exact ties on some channels
+    got_bits = run_conv(bk, x, w, thr, s, p, engine)
+    assert np.array_equal(got_bits, oracle.threshold(want, thr))
+    thr = plant_extreme_thresholds(thr, K)
     got_bits = run_conv(bk, x, w, thr, s, p, engine)
     assert np.array_equal(got_bits, oracle.threshold(want, thr))
 
@@ -146,6 +159,13 @@ def test_gemm_int32_and_fused(bk, oracle, shape, engine):
         thr = synth.thresholds(rng, K, N)
         raw, ob = guard_alloc(M * N // 8)
         call_or_skip(bk, engine, lambda: bk.bcnn_gemm_b1_fused(Ab, Wb, dev(thr), ob, M, N, K, engine=bk.ENGINES[engine]))
+        torch.cuda.synchronize()
+        check_guards(raw, M * N // 8)
+        assert np.array_equal(synth.unpack_bits(ob.cpu().numpy().reshape(M, N // 8)), oracle.threshold(want, thr))
+        thr = plant_extreme_thresholds(thr, K)
+        thr[::4] = want[M // 2, ::4]                    # ties
+        raw, ob = guard_alloc(M * N // 8)
+        bk.bcnn_gemm_b1_fused(Ab, Wb, dev(thr), ob, M, N, K, engine=bk.ENGINES[engine])
         torch.cuda.synchronize()
         check_guards(raw, M * N // 8)
         assert np.array_equal(synth.unpack_bits(ob.cpu().numpy().reshape(M, N // 8)), oracle.threshold(want, thr))
@@ -290,6 +310,28 @@ def test_errors_launch_nothing(bk):
         bk.bcnn_gemm_b1_fused(a, a, None, a, 8, 32, 32)
     torch.cuda.synchronize()
     assert int(a.sum()) == 0
+    assert bk.bcnn_device_error() == 0
+
+
+def test_bounded_wait_runs_out_and_is_reported(bk, oracle):
+    # failure detection without a fault: a wait that nothing satisfies gives up after its poll limit, the kernel
+    # frees its tensor memory and ends normally, the error word carries the code until it is read, and the context
+    # (tensor memory included: the next tcgen05 kernel allocates all of it) stays usable
+    assert bk.bcnn_device_error() == 0
+    bk.bcnn_selftest_wait_timeout(256)
+    torch.cuda.synchronize()                               # the kernel ended by itself
+    st, code = bk.bcnn_device_status()
+    assert st == bk.ERR_TIMEOUT and code == bk.SELFTEST_TIMEOUT_CODE
+    assert "self-test" in bk.status_string(code)
+    assert bk.bcnn_device_status() == (bk.OK, 0)           # reading cleared it
+    bk.bcnn_selftest_wait_timeout(1)
+    assert bk.bcnn_device_error() == bk.SELFTEST_TIMEOUT_CODE and bk.bcnn_device_error() == 0
+    # a normal convolution on both tcgen05 engines right after: bit-exact, no error
+    rng = np.random.default_rng(31337)
+    x, w = synth.pm1(rng, (2, 12, 12, 64)), synth.pm1(rng, (64, 3, 3, 64))
+    want = oracle.conv2d(x, w, 1, 1)
+    for engine in ("tc_ws", "tc_i8"):
+        assert np.array_equal(run_conv(bk, x, w, None, 1, 1, engine), want)
     assert bk.bcnn_device_error() == 0
 
 
