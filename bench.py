@@ -797,7 +797,7 @@ def run_paper1x1(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--mode", default="bench", choices=["bench", "sweep", "paper1x1"])
-    ap.add_argument("--engines", default="auto,lop3,mma_b1,tc_i8,mma_s8,tc_ws")
+    ap.add_argument("--engines", default="auto,lop3,mma_b1,tc_i8,mma_s8,tc_ws,tc_pw")
     ap.add_argument("--sweep-set", default="all", choices=["gemm", "conv", "all"])
     ap.add_argument("--only", default="", help="sweep mode: run only shapes whose label contains this text")
     ap.add_argument("--outs", default="int32,fused", help="sweep mode: output kinds to run")

@@ -58,7 +58,9 @@ typedef enum bcnn_engine {
     BCNN_ENGINE_MMA_B1 = 2, /* warp-level mma.sync m16n8k256 .b1 AND + popcount         */
     BCNN_ENGINE_TC_I8 = 3,  /* sign bits expanded to bytes in shared memory, tcgen05 kind::i8, TMEM accumulators */
     BCNN_ENGINE_MMA_S8 = 4, /* sign bits expanded to bytes in registers, warp-level mma.sync 8-bit (narrow layers) */
-    BCNN_ENGINE_TC_WS = 5   /* tcgen05 kind::i8 with the expanded weight tile resident in shared memory (C_out <= 128) */
+    BCNN_ENGINE_TC_WS = 5,  /* tcgen05 kind::i8 with the expanded weight tile resident in shared memory (C_out <= 128) */
+    BCNN_ENGINE_TC_PW = 6   /* tcgen05 kind::i8 for pointwise layers (1x1, stride 1, no padding; GEMMs) with K <= 128 and
+                               C_out <= 128, packed output: rows bulk-copied in chunks, one hand-over per chunk */
 } bcnn_engine;
 
 /*

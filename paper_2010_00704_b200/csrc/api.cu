@@ -74,6 +74,8 @@ int make_conv_problem(ConvProblem &p, const void *x, const void *w, const int32_
 }
 
 // Measured on B200 (bench.py --mode sweep):
+//   * pointwise layers (1x1, stride 1, no padding; GEMMs) with K <= 128 and C_out <= 128, packed output: pointwise
+//     tcgen05 engine (memory-bound shapes: rows bulk-copied in chunks, one hand-over per chunk);
 //   * C_out >= 256, or weights too large to keep expanded in shared memory: streaming tcgen05 engine;
 //   * 1x1 layer with C_in = 32 and C_out <= 32 (one XOR + popcount per output): CUDA-core pointwise kernel;
 //   * C_out <= 128 with K >= 64, and wider layers with K <= 1152 and M >= 32768 (in 128-channel slices):
@@ -82,6 +84,7 @@ int make_conv_problem(ConvProblem &p, const void *x, const void *w, const int32_
 //   * the single-bit mma.sync and CUDA-core engines never win and serve as fallbacks.
 int auto_engine(const ConvProblem &p)
 {
+    if (conv_tc_pw_supports(p)) return BCNN_ENGINE_TC_PW;
     if (conv_lop3_pointwise_k32(p)) return BCNN_ENGINE_LOP3;
     if (p.C_out <= 128 && p.K >= 64 && conv_tc_ws_supports(p)) return BCNN_ENGINE_TC_WS;
     // wider layers in slices of 128 output channels: ahead of the streaming engine while K is short and there are
@@ -107,6 +110,8 @@ int dispatch(int engine, const ConvProblem &p, cudaStream_t stream)
         return launch_conv_mma_s8(p, stream);
     case BCNN_ENGINE_TC_WS:
         return launch_conv_tc_ws(p, stream);
+    case BCNN_ENGINE_TC_PW:
+        return launch_conv_tc_pw(p, stream);
     default:
         return BCNN_ERR_UNSUPPORTED;
     }
@@ -293,6 +298,12 @@ const char *bcnn_status_string(int status)
     case 111: return "device wait timed out: weight-stationary tcgen05 engine, producer waiting for a free ring slot";
     case 112: return "device wait timed out: weight-stationary tcgen05 engine, control warp waiting for a full slot or a free accumulator";
     case 113: return "device wait timed out: weight-stationary tcgen05 engine, epilogue waiting for an accumulator";
+    case 121: return "device wait timed out: pointwise tcgen05 engine, loader waiting for a free ring stage";
+    case 122: return "device wait timed out: pointwise tcgen05 engine, producer waiting for a chunk's rows";
+    case 123: return "device wait timed out: pointwise tcgen05 engine, issuer waiting for a slot's expanded rows";
+    case 124: return "device wait timed out: pointwise tcgen05 engine, epilogue waiting for a chunk's accumulators";
+    case 125: return "device wait timed out: pointwise tcgen05 engine, producer waiting for a slot's previous MMAs";
+    case 126: return "device wait timed out: pointwise tcgen05 engine, issuer waiting for a slot's accumulators";
     case BCNN_SELFTEST_TIMEOUT_CODE: return "device wait timed out: self-test (expected)";
     default: return status > 0 ? "device-side error code" : "unknown status";
     }

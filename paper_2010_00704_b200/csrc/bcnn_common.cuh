@@ -77,6 +77,8 @@ int launch_conv_mma_s8(const ConvProblem &p, cudaStream_t stream);
 bool conv_mma_s8_supports(const ConvProblem &p);
 int launch_conv_tc_ws(const ConvProblem &p, cudaStream_t stream);
 bool conv_tc_ws_supports(const ConvProblem &p);
+int launch_conv_tc_pw(const ConvProblem &p, cudaStream_t stream);
+bool conv_tc_pw_supports(const ConvProblem &p);
 int launch_conv_tc_i8(const ConvProblem &p, cudaStream_t stream);
 bool conv_tc_i8_supports(const ConvProblem &p);
 int launch_selftest_wait_timeout(int polls, cudaStream_t stream);

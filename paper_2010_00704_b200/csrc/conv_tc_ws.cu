@@ -249,8 +249,10 @@ conv_tc_ws_kernel(const ConvProblem p)
             if (lane == 0 && alive) alive = mbar_wait(tempty_bar(buf), buf_phase, abort_flag, p.err, ERR_MMA_TIMEOUT);
             for (int kt = 0; kt < ktiles; ++kt) {
                 if (lane == 0 && alive) alive = mbar_wait(full_bar(s), ring_phase, abort_flag, p.err, ERR_MMA_TIMEOUT);
-                __syncwarp();
-                asm volatile("bar.arrive %0, 64;" ::"r"(1 + s) : "memory");
+                // after a time-out: bar.sync, which pairs every release with one wait of the issuer (two bar.arrive in a
+                // row on one barrier would complete it without the issuer)
+                if (__shfl_sync(0xffffffffu, alive ? 1 : 0, 0)) asm volatile("bar.arrive %0, 64;" ::"r"(1 + s) : "memory");
+                else asm volatile("bar.sync %0, 64;" ::"r"(1 + s) : "memory");
                 if (++s == STAGES) { s = 0; ring_phase ^= 1u; }
             }
             if (++buf == NBUF) { buf = 0; buf_phase ^= 1u; }
