@@ -104,13 +104,15 @@ __host__ __device__ constexpr int channel_of_column(int c)
 }
 
 // 64 accumulator columns of this warp's 32 rows as packed 16-bit halves: register i = columns 2i (low) and 2i + 1.
+// The loads below do NOT wait: several are issued in a row, then tc_wait_ld(), then pin_regs() on every destination
+// array - an empty volatile asm that takes the registers as read-write operands, so that no use of them can be
+// scheduled ahead of the wait.
 __device__ __forceinline__ void tc_ld64_pack16(uint32_t taddr, uint32_t (&v)[32])
 {
     asm volatile(
         "tcgen05.ld.sync.aligned.32x32b.x32.pack::16b.b32 "
         "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
-        "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];\n\t"
-        "tcgen05.wait::ld.sync.aligned;"
+        "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
         : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
           "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
           "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
@@ -122,12 +124,55 @@ __device__ __forceinline__ void tc_ld32_pack16(uint32_t taddr, uint32_t (&v)[16]
 {
     asm volatile(
         "tcgen05.ld.sync.aligned.32x32b.x16.pack::16b.b32 "
-        "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];\n\t"
-        "tcgen05.wait::ld.sync.aligned;"
+        "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
         : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
           "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
         : "r"(taddr) : "memory");
 }
+__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+__device__ __forceinline__ void pin_regs(uint32_t (&v)[16])
+{
+    asm volatile("" : "+r"(v[0]), "+r"(v[1]), "+r"(v[2]), "+r"(v[3]), "+r"(v[4]), "+r"(v[5]), "+r"(v[6]), "+r"(v[7]),
+                      "+r"(v[8]), "+r"(v[9]), "+r"(v[10]), "+r"(v[11]), "+r"(v[12]), "+r"(v[13]), "+r"(v[14]), "+r"(v[15]) :: "memory");
+}
+__device__ __forceinline__ void pin_regs(uint32_t (&v)[32])
+{
+    asm volatile("" : "+r"(v[0]), "+r"(v[1]), "+r"(v[2]), "+r"(v[3]), "+r"(v[4]), "+r"(v[5]), "+r"(v[6]), "+r"(v[7]),
+                      "+r"(v[8]), "+r"(v[9]), "+r"(v[10]), "+r"(v[11]), "+r"(v[12]), "+r"(v[13]), "+r"(v[14]), "+r"(v[15]),
+                      "+r"(v[16]), "+r"(v[17]), "+r"(v[18]), "+r"(v[19]), "+r"(v[20]), "+r"(v[21]), "+r"(v[22]), "+r"(v[23]),
+                      "+r"(v[24]), "+r"(v[25]), "+r"(v[26]), "+r"(v[27]), "+r"(v[28]), "+r"(v[29]), "+r"(v[30]), "+r"(v[31]) :: "memory");
+}
+
+// Waits of this engine: hand-overs are on the critical path of a slot's cycle, so the waiter sleeps only briefly
+// between polls (a failed try_wait returns at once: measured, polling without any sleep more than doubled the
+// instructions the SM executes; the shared helpers' 100 ns is a fifth of a slot's cycle here).
+// Bounded by elapsed clock cycles (about two seconds), checked every 64 polls together with the CTA's abort flag.
+constexpr long long PW_WAIT_CYCLES = 4000000000LL;
+constexpr uint32_t PW_SLEEP_NS = 32;
+static __device__ __noinline__ bool pw_wait_slow(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *err, int code)
+{
+    const long long t0 = clock64();
+    for (uint32_t it = 1;; ++it) {
+        __nanosleep(PW_SLEEP_NS);
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((it & 63u) == 0u) {
+            if (*abort_flag) return false;
+            if (clock64() - t0 > PW_WAIT_CYCLES) break;
+        }
+    }
+    *abort_flag = 1;
+    if (err) atomicCAS(err, 0, code);
+    return false;
+}
+// whole-warp wait (every lane polls; the verdict is a vote)
+__device__ __forceinline__ bool pw_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *err, int code)
+{
+    bool ok = mbar_try_wait(bar, parity);
+    if (__all_sync(0xffffffffu, ok)) return true;
+    if (!ok) ok = pw_wait_slow(bar, parity, abort_flag, err, code);
+    return __all_sync(0xffffffffu, ok);
+}
+
 // Output word of a 32-column block from its 16 packed registers: bit = (accumulator >= 0).  PRMT in sign-replication
 // mode turns the two halves of two registers into four bytes 0x00 / 0xFF; step s keeps bit s of every byte.
 __device__ __forceinline__ uint32_t sign_word(const uint32_t *r)
@@ -257,8 +302,8 @@ conv_tc_pw_kernel(const ConvProblem p)
         uint32_t phase = 0;
         for (int j = slot; j < my_chunks; j += NSLOT) {
             // the epilogue has read the slot's previous accumulators (nothing to wait for the first time round)
-            if (j >= NSLOT && !mbar_wait_warp(acc_free(slot), phase ^ 1u, abort_flag, p.err, ERR_PW_ACC_TIMEOUT)) break;
-            if (!mbar_wait_warp(a_full(slot), phase, abort_flag, p.err, ERR_PW_ISSUER_TIMEOUT)) break;
+            if (j >= NSLOT && !pw_wait(acc_free(slot), phase ^ 1u, abort_flag, p.err, ERR_PW_ACC_TIMEOUT)) break;
+            if (!pw_wait(a_full(slot), phase, abort_flag, p.err, ERR_PW_ISSUER_TIMEOUT)) break;
             tc_fence_after();
             if (elect_one()) {
 #pragma unroll
@@ -287,7 +332,7 @@ conv_tc_pw_kernel(const ConvProblem p)
             const long row0 = ((long)blockIdx.x + (long)b * gridDim.x) * C::BLOCK_ROWS;
             const long rows = min((long)C::BLOCK_ROWS, (long)p.M - row0);
             const uint32_t bytes = (uint32_t)rows * KW * 4u;
-            if (!mbar_wait_warp(load_empty(stage), phase, abort_flag, p.err, ERR_PW_LOADER_TIMEOUT)) break;
+            if (!pw_wait(load_empty(stage), phase, abort_flag, p.err, ERR_PW_LOADER_TIMEOUT)) break;
             const uint32_t dst = ring + (uint32_t)stage * C::BLOCK_BYTES;
             const uint32_t *src = p.x + row0 * KW;
             if ((bytes & 15u) == 0u) {
@@ -310,7 +355,7 @@ conv_tc_pw_kernel(const ConvProblem p)
         if (*abort_flag) {
             const int first = issued > NBLK ? issued - NBLK : 0;
             for (int b = first; b < issued; ++b)
-                mbar_wait_warp(load_full(b % NBLK), (uint32_t)(b / NBLK) & 1u, abort_flag, nullptr, 0);
+                pw_wait(load_full(b % NBLK), (uint32_t)(b / NBLK) & 1u, abort_flag, nullptr, 0);
         }
     } else if (warp >= C::FIRST_EPILOGUE_WARP) {
         // ------------------------------------------------------------------ epilogue of slot (warp - first) / 4
@@ -321,35 +366,39 @@ conv_tc_pw_kernel(const ConvProblem p)
         uint32_t phase = 0;
         for (int j = slot; j < my_chunks; j += NSLOT) {
             const long row_w = chunk_row0(j) + quad * 32 + lane;                 // this thread's row in tile 0
-            bool alive = mbar_wait(mma_done(slot), phase, abort_flag, p.err, ERR_PW_EPILOGUE_TIMEOUT);
-            alive = __all_sync(0xffffffffu, alive && !*abort_flag);
-            if (!alive) break;
+            if (!pw_wait(mma_done(slot), phase, abort_flag, p.err, ERR_PW_EPILOGUE_TIMEOUT)) break;
             tc_fence_after();
             phase ^= 1u;
+            // all of the chunk's accumulators -> registers, one wait, and the slot goes back to the issuer before
+            // any bit is gathered
+            constexpr int NR = BN == 32 ? 16 : 32;                       // registers per load
+            constexpr int NL = BN == 32 ? 1 : BN / 64;                   // loads per tile
+            uint32_t r[T * NL][NR];
+#pragma unroll
+            for (int t = 0; t < T; ++t) {
+                if constexpr (BN == 32) {
+                    tc_ld32_pack16(t_lane + (uint32_t)(t * BN), r[t]);
+                } else {
+#pragma unroll
+                    for (int h = 0; h < NL; ++h) tc_ld64_pack16(t_lane + (uint32_t)(t * BN + h * 64), r[t * NL + h]);
+                }
+            }
+            tc_wait_ld();
+#pragma unroll
+            for (int q = 0; q < T * NL; ++q) pin_regs(r[q]);
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(acc_free(slot));
 #pragma unroll
             for (int t = 0; t < T; ++t) {
                 uint32_t words[BN / 32];
                 if constexpr (BN == 32) {
-                    uint32_t r[16];
-                    tc_ld32_pack16(t_lane + (uint32_t)(t * BN), r);
-                    if (t == T - 1) {                                     // all of the slot's accumulators are in registers
-                        tc_fence_before();
-                        __syncwarp();
-                        if (lane == 0) mbar_arrive(acc_free(slot));
-                    }
-                    words[0] = sign_word(r);
+                    words[0] = sign_word(r[t]);
                 } else {
 #pragma unroll
-                    for (int h = 0; h < BN / 64; ++h) {
-                        uint32_t r[32];
-                        tc_ld64_pack16(t_lane + (uint32_t)(t * BN + h * 64), r);
-                        if (t == T - 1 && h == BN / 64 - 1) {
-                            tc_fence_before();
-                            __syncwarp();
-                            if (lane == 0) mbar_arrive(acc_free(slot));
-                        }
-                        words[2 * h] = sign_word(r);
-                        words[2 * h + 1] = sign_word(r + 16);
+                    for (int h = 0; h < NL; ++h) {
+                        words[2 * h] = sign_word(r[t * NL + h]);
+                        words[2 * h + 1] = sign_word(r[t * NL + h] + 16);
                     }
                 }
                 const long m = row_w + (long)t * BM;
@@ -378,7 +427,7 @@ conv_tc_pw_kernel(const ConvProblem p)
         uint32_t phase = 0;
         for (int j = slot; j < my_chunks; j += NSLOT) {
             const int blk = j / G, stage = blk % NBLK;
-            if (!mbar_wait_warp(load_full(stage), (uint32_t)(blk / NBLK) & 1u, abort_flag, p.err, ERR_PW_PRODUCER_TIMEOUT)) break;
+            if (!pw_wait(load_full(stage), (uint32_t)(blk / NBLK) & 1u, abort_flag, p.err, ERR_PW_PRODUCER_TIMEOUT)) break;
             const uint32_t src = ring + (uint32_t)stage * C::BLOCK_BYTES + (uint32_t)(j % G) * C::CHUNK_BYTES + (uint32_t)row * (KW * 4u);
             uint32_t wds[T][KW];
 #pragma unroll
@@ -397,23 +446,25 @@ conv_tc_pw_kernel(const ConvProblem p)
             }
             __syncwarp();
             mbar_arrive_pred(load_empty(stage), lane0);           // (the stage may be refilled once all its chunks have been read)
+            // expanded rows in registers first; only the stores wait for the slot
+            uint32_t v[T][8 * KW];
+#pragma unroll
+            for (int t = 0; t < T; ++t)
+#pragma unroll
+                for (int e = 0; e < KW; ++e) expand_a(wds[t][e], &v[t][8 * e]);
             // the MMAs of the slot's previous chunk have read its activation columns
-            if (j >= NSLOT && !mbar_wait_warp(mma_done(slot), phase ^ 1u, abort_flag, p.err, ERR_PW_SLOT_TIMEOUT)) break;
+            if (j >= NSLOT && !pw_wait(mma_done(slot), phase ^ 1u, abort_flag, p.err, ERR_PW_SLOT_TIMEOUT)) break;
             tc_fence_after();
 #pragma unroll
             for (int t = 0; t < T; ++t) {
                 const uint32_t taddr = t_lane + (uint32_t)(t * C::A_COLS);
                 if constexpr (KW == 4) {
-                    uint32_t v[32];
-#pragma unroll
-                    for (int e = 0; e < 4; ++e) expand_a(wds[t][e], &v[8 * e]);
-                    tc_st32_nowait(taddr, v);
+                    tc_st32_nowait(taddr, v[t]);
                 } else {
 #pragma unroll
                     for (int e = 0; e < KW; ++e) {
-                        uint32_t v[8];
-                        expand_a(wds[t][e], v);
-                        tc_st8_nowait(taddr + 8u * e, v);
+                        const uint32_t (&v8)[8] = *reinterpret_cast<const uint32_t (*)[8]>(&v[t][8 * e]);
+                        tc_st8_nowait(taddr + 8u * e, v8);
                     }
                 }
             }
