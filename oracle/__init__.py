@@ -2,10 +2,12 @@
 
 Nothing in the product package imports this.  Only the tests, the smoke check and
 the CPU-baseline leg of the benchmark may use it.  The arithmetic lives in plain C
-(``bcnn_oracle.c``: the definition, on unpacked int8 +-1 tensors; ``bcnn_checker.c``:
+(``bcnn_oracle.c``: the definition, on unpacked int8 +-1 tensors; ``bcnn_block_oracle.c``:
+the rest of the paper's building block - parallel binary branches, depth-wise 3x3 module,
+average pooling, global pooling and the fully connected layer; ``bcnn_checker.c``:
 a separately written bit-packed checker for full-size coverage, trusted only
 through the tests that prove it equal to the definition).  This module compiles
-those two files with gcc and marshals numpy arrays; it holds no arithmetic of the
+those files with gcc and marshals numpy arrays; it holds no arithmetic of the
 method itself.
 
 Parity pins (see tests/test_oracle_pins.py): closed forms for constant inputs
@@ -17,7 +19,11 @@ norm, identity, PReLU, fp16 store, next sign) a case worked by hand, the fp16
 round-to-even ties, the sign-of-the-stored-value rule, the reduction to the integer
 threshold and the elementwise numpy restatement.  The paper prints no worked
 numeric example of a convolution, so beyond those pins parity is unpinned by the
-paper itself.
+paper itself.  The block pieces are pinned in tests/test_block_oracle_pins.py: the branch
+module against the single-branch function, a hand-worked two-branch case and the order
+of summation; the shifted-branch form of an F x F convolution against the textbook zero-
+padded convolution and against the -1-padded one; depth-wise convolution, pooling and the
+fully connected layer against closed forms and the float64 library routines.
 """
 from __future__ import annotations
 
@@ -30,7 +36,8 @@ import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _LIB_PATH = os.path.join(_HERE, "libbcnn_oracle.so")
-_SOURCES = [os.path.join(_HERE, "bcnn_oracle.c"), os.path.join(_HERE, "bcnn_checker.c")]
+_SOURCES = [os.path.join(_HERE, "bcnn_oracle.c"), os.path.join(_HERE, "bcnn_block_oracle.c"),
+            os.path.join(_HERE, "bcnn_checker.c")]
 _lock = threading.Lock()
 _lib = None
 
@@ -186,6 +193,116 @@ def conv_module(acc: np.ndarray, scale, shift, identity, slope, next_bias=None, 
     _load().oracle_conv_module(_ptr(acc), _ptr(scale), _ptr(shift), iptr, _ptr(slope), nptr, _ptr(y),
                                None if s is None else _ptr(s), ctypes.c_long(rows), ctypes.c_long(N))
     return y, s
+
+
+def conv_module_branches(accs, scales, shifts, identity, slope, next_bias=None, want_sign: bool = True):
+    """Module with P parallel binary branches (Section 4.2.1, Figure 4 bottom): accs int32 [P, ..., N], scales and
+    shifts fp32 [P, N]; the rest as ``conv_module``.  Returns (y float16, s int8 or None)."""
+    accs = _c(accs, np.int32)
+    P, N = accs.shape[0], accs.shape[-1]
+    scales, shifts, slope = _c(scales, np.float32), _c(shifts, np.float32), _c(slope, np.float32)
+    assert scales.shape == (P, N) and shifts.shape == (P, N) and slope.shape == (N,)
+    iptr = None
+    if identity is not None:
+        identity = _c(identity, np.float16)
+        assert identity.shape == accs.shape[1:]
+        iptr = _ptr(identity)
+    nptr = None
+    if next_bias is not None:
+        next_bias = _c(next_bias, np.float32)
+        assert next_bias.shape == (N,)
+        nptr = _ptr(next_bias)
+    y = np.empty(accs.shape[1:], dtype=np.float16)
+    s = np.empty(accs.shape[1:], dtype=np.int8) if want_sign else None
+    rows = y.size // N if N else 0
+    _load().oracle_conv_module_branches(_ptr(accs), _ptr(scales), _ptr(shifts), iptr, _ptr(slope), nptr, _ptr(y),
+                                        None if s is None else _ptr(s), ctypes.c_long(rows), ctypes.c_long(N), P)
+    return y, s
+
+
+def shifted_branch_accs(x_real, biases, ws, kh: int, kw: int, pad_zero_contribution: bool = False):
+    """The P = kh*kw branch convolutions that stand for a binary kh x kw convolution (Section 4.2.1, last paragraph):
+    branch p = (r, t) sees the real map shifted by (r - (kh-1)/2, t - (kw-1)/2) with ZERO padding, adds its own bias,
+    takes the sign and runs its own binary 1x1 convolution.  Steps, in the paper's order, from existing pieces:
+    shift + zero pad (array slicing), ``binarize``, ``conv2d`` (1x1).
+      x_real float16 [B,H,W,C_in]; biases fp32 [P,C_in]; ws int8 [P,C_out,C_in] (+-1).
+    Returns (accs int32 [P,B,H,W,C_out], inside bool [P,H,W]).  With ``pad_zero_contribution`` a branch whose pixel
+    lies outside the image contributes 0 instead of the convolution of sign(0 + bias) (the other reading)."""
+    x_real = _c(x_real, np.float16)
+    B, H, W, C_in = x_real.shape
+    P = kh * kw
+    biases = _c(biases, np.float32)
+    ws = _c(ws, np.int8)
+    assert biases.shape == (P, C_in) and ws.shape[0] == P and ws.shape[2] == C_in
+    accs, insides = [], []
+    for p in range(P):
+        r, t = divmod(p, kw)
+        dy, dx = r - (kh - 1) // 2, t - (kw - 1) // 2
+        shifted = np.zeros_like(x_real)
+        inside = np.zeros((H, W), dtype=bool)
+        h0, h1 = max(0, -dy), min(H, H - dy)
+        w0, w1 = max(0, -dx), min(W, W - dx)
+        if h1 > h0 and w1 > w0:
+            shifted[:, h0:h1, w0:w1, :] = x_real[:, h0 + dy:h1 + dy, w0 + dx:w1 + dx, :]
+            inside[h0:h1, w0:w1] = True
+        bits = binarize(shifted.astype(np.float32), biases[p], 1)
+        acc = conv2d(bits, ws[p][:, None, None, :], 1, 0)
+        if pad_zero_contribution:
+            acc = acc * inside[None, :, :, None].astype(np.int32)
+        accs.append(acc)
+        insides.append(inside)
+    return np.stack(accs), np.stack(insides)
+
+
+def dwconv3x3_module(x, w, scale, shift, slope, R: int = 1, S: int = 1) -> np.ndarray:
+    """Real depth-wise 3x3 convolution (stride S, zero padding 1), batch norm, PReLU (Section 4.2.1), with channel
+    replication R (Section 4.2.2).  x float16 [B,H,W,C_in]; w fp32 [C,3,3]; per-channel fp32 [C]; C = R*C_in.
+    fp64 arithmetic, one rounding to float16."""
+    x = _c(x, np.float16)
+    B, H, W, C_in = x.shape
+    C = C_in * R
+    w, scale, shift, slope = _c(w, np.float32), _c(scale, np.float32), _c(shift, np.float32), _c(slope, np.float32)
+    assert w.shape == (C, 3, 3) and scale.shape == (C,) and shift.shape == (C,) and slope.shape == (C,)
+    OH, OW = (H + 2 - 3) // S + 1, (W + 2 - 3) // S + 1
+    y = np.empty((B, OH, OW, C), dtype=np.float16)
+    _load().oracle_dwconv3x3_module(_ptr(x), _ptr(w), _ptr(scale), _ptr(shift), _ptr(slope), _ptr(y), B, H, W, C_in, R, S)
+    return y
+
+
+def avgpool(x, S: int, R: int = 1) -> np.ndarray:
+    """S x S / S average pooling (Section 4.2.3) with channel replication R; float16 in and out, fp64 mean."""
+    x = _c(x, np.float16)
+    B, H, W, C_in = x.shape
+    assert H % S == 0 and W % S == 0
+    y = np.empty((B, H // S, W // S, C_in * R), dtype=np.float16)
+    _load().oracle_avgpool(_ptr(x), _ptr(y), B, H, W, C_in, R, S)
+    return y
+
+
+def gap(x) -> np.ndarray:
+    """Global average pooling (Section 4.1): float16 [B,H,W,C] -> float64 [B,C]."""
+    x = _c(x, np.float16)
+    B, H, W, C = x.shape
+    out = np.empty((B, C), dtype=np.float64)
+    _load().oracle_gap(_ptr(x), _ptr(out), B, ctypes.c_long(H * W), C)
+    return out
+
+
+def fc(pooled, w, bias=None) -> np.ndarray:
+    """Fully connected layer (Section 4.1): pooled float64 [B,C], w fp32 [N,C], bias fp32 [N] -> float64 [B,N]."""
+    pooled = _c(pooled, np.float64)
+    w = _c(w, np.float32)
+    B, C = pooled.shape
+    N = w.shape[0]
+    assert w.shape == (N, C)
+    bptr = None
+    if bias is not None:
+        bias = _c(bias, np.float32)
+        assert bias.shape == (N,)
+        bptr = _ptr(bias)
+    out = np.empty((B, N), dtype=np.float64)
+    _load().oracle_fc(_ptr(pooled), _ptr(w), bptr, _ptr(out), B, C, N)
+    return out
 
 
 # ---- bit-packed checker (not the oracle; proven equal to it by the CPU tests) ----
