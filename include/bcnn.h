@@ -139,6 +139,59 @@ int bcnn_conv2d_b1_module(const void *x_bits, const void *w_bits, const float *b
                           int kh, int kw, int stride, int pad, void *stream);
 
 /*
+ * Convolution module with P parallel binary residual branches (Section 4.2.1, Figure 4 bottom: each branch has its own
+ * learned bias - hence its own binarization -, its own binary weights and its own batch norm; the branches are summed
+ * before the identity addition and PReLU), in one pass:
+ *   dot_p = binary 1x1 convolution of branch p's sign channels with branch p's weights
+ *   t_p = dot_p * bn_scale[p][co] + bn_shift[p][co];   t = ((t_0 + t_1) + t_2) + ...        (branch order, fp32)
+ *   u = t + identity;  r = (u >= 0) ? u : prelu_slope[co] * u;  y_real = fp16(r);  y bit = (y_real + next_bias[co] >= 0)
+ * one fp32 operation per step as in bcnn_conv2d_b1_module (which this call equals for P = 1, kh = kw = 1).
+ *   x_bits   device, packed NHWC [B][H][W][P * C_in]: branch p's signs are channels [p*C_in, (p+1)*C_in) of a pixel,
+ *            i.e. the output of ONE bcnn_pack call with R = P and the P branch biases concatenated
+ *   w_bits   device, packed [P][C_out][C_in];   bn_scale, bn_shift  device fp32 [P][C_out]
+ * With kh * kw > 1 the branches are the taps of a binary kh x kw convolution (last paragraph of Section 4.2.1: P = kh*kw
+ * branches, each on the real map shifted to its tap with zero padding applied BEFORE the branch's bias and sign); then
+ * P must equal kh * kw, branch p = (r, t) reads pixel (h + r - (kh-1)/2, w + t - (kw-1)/2), and where that pixel lies
+ * outside the image its dot_p is pad_dot[p][co] - the caller passes sum_ci sign(0 + bias_p[ci]) * w_p[co][ci] for the
+ * paper's padding, or NULL (0) for a tap that contributes nothing.  Stride 1, output H x W.
+ *   pad_dot  device int32 [P][C_out] or NULL;  identity, prelu_slope, next_bias, y_real, y_bits as in
+ *   bcnn_conv2d_b1_module (identity and y_real may be the same buffer).  C_in % 32 == 0, C_out % 32 == 0.
+ */
+int bcnn_conv2d_b1_branches(const void *x_bits, const void *w_bits, const float *bn_scale, const float *bn_shift,
+                            const int32_t *pad_dot, const void *identity, const float *prelu_slope, const float *next_bias,
+                            void *y_real, void *y_bits, int B, int H, int W, int C_in, int C_out, int P, int kh, int kw,
+                            void *stream);
+
+/*
+ * The 3x3 convolution module (Section 4.2.1: real depth-wise 3x3 convolution for spatial mixing, batch norm, PReLU), with
+ * stride S (Section 4.2.3) and channel replication by bookkeeping (Section 4.2.2: output channel c reads input channel
+ * c mod C_in; nothing is copied):
+ *   conv = sum_{r,t} xpad[oh*S - 1 + r][ow*S - 1 + t][c mod C_in] * w[c][r][t],  xpad = 0 outside the image
+ *   y_real = fp16(PReLU(conv * bn_scale[c] + bn_shift[c]));   y bit = (y_real + next_bias[c] >= 0)   (optional)
+ * fp32 arithmetic on fp16 storage.  x device fp16 NHWC [B][H][W][C_in]; w device fp32 [C][3][3], C = R * C_in;
+ * y_real device fp16 [B][OH][OW][C], OH = (H - 1) / S + 1; y_bits device packed [B][OH][OW][C] or NULL (then next_bias
+ * is ignored); next_bias may be NULL (0).  C_in % 8 == 0; C % 32 == 0 when y_bits is given.
+ */
+int bcnn_dwconv3x3_module(const void *x, const float *w, const float *bn_scale, const float *bn_shift, const float *prelu_slope,
+                          const float *next_bias, void *y_real, void *y_bits, int B, int H, int W, int C_in, int R, int S,
+                          void *stream);
+
+/*
+ * S x S average pooling with stride S on the identity path of a down-sampling block (Section 4.2.3), with the same
+ * channel replication: y[b][oh][ow][c] = fp16(mean of the S x S window of x[..][c mod C_in]).  H % S == 0, W % S == 0,
+ * C_in % 8 == 0.  S = 1 with R > 1 is plain replication of a map that a consumer needs materialised.
+ */
+int bcnn_avgpool(const void *x, void *y, int B, int H, int W, int C_in, int R, int S, void *stream);
+
+/*
+ * Head (Section 4.1, Figure 2; last rows of Table 1): global average pooling, pooled[b][c] = mean over the H*W pixels of
+ * x (fp16 NHWC) as fp32 [B][C], and the fully connected layer logits[b][n] = sum_c pooled[b][c] * w[n][c] + bias[n]
+ * (w fp32 [N][C], bias fp32 [N] or NULL, logits fp32 [B][N]).  C % 8 == 0.
+ */
+int bcnn_gap(const void *x, float *pooled, int B, int H, int W, int C, void *stream);
+int bcnn_fc(const float *pooled, const float *w, const float *bias, float *logits, int B, int C, int N, void *stream);
+
+/*
  * Fused stem: bcnn_pack followed by the first binary 1x1 convolution with its threshold epilogue, without
  * writing the packed sign tensor in between (Section 4.1: the stem uses the same block, so even the first
  * convolution is binary; Table 1 "stem replicate": 4 real channels replicated 8x to 32 sign channels;

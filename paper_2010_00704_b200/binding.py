@@ -21,6 +21,7 @@ ENGINES = {"auto": ENGINE_AUTO, "lop3": ENGINE_LOP3, "mma_b1": ENGINE_MMA_B1, "t
 
 EXPORTS = (
     "bcnn_pack", "bcnn_stem_fused", "bcnn_gemm_b1", "bcnn_gemm_b1_fused", "bcnn_conv2d_b1", "bcnn_conv2d_b1_fused", "bcnn_conv2d_b1_module",
+    "bcnn_conv2d_b1_branches", "bcnn_dwconv3x3_module", "bcnn_avgpool", "bcnn_gap", "bcnn_fc",
     "bcnn_conv2d_b1_engine", "bcnn_gemm_b1_engine", "bcnn_auto_engine", "bcnn_device_error", "bcnn_device_status",
     "bcnn_workspace_bytes", "bcnn_selftest_wait_timeout", "bcnn_status_string", "bcnn_version",
 )
@@ -53,6 +54,11 @@ def load() -> ctypes.CDLL:
         lib.bcnn_conv2d_b1.argtypes = [vp, vp, vp] + [i32] * 9 + [vp]
         lib.bcnn_conv2d_b1_fused.argtypes = [vp, vp, vp, vp] + [i32] * 9 + [vp]
         lib.bcnn_conv2d_b1_module.argtypes = [vp] * 9 + [i32] * 9 + [vp]
+        lib.bcnn_conv2d_b1_branches.argtypes = [vp] * 10 + [i32] * 8 + [vp]
+        lib.bcnn_dwconv3x3_module.argtypes = [vp] * 8 + [i32] * 6 + [vp]
+        lib.bcnn_avgpool.argtypes = [vp, vp] + [i32] * 6 + [vp]
+        lib.bcnn_gap.argtypes = [vp, vp] + [i32] * 4 + [vp]
+        lib.bcnn_fc.argtypes = [vp] * 4 + [i32] * 3 + [vp]
         lib.bcnn_conv2d_b1_engine.argtypes = [i32, vp, vp, vp, vp] + [i32] * 9 + [vp]
         lib.bcnn_gemm_b1_engine.argtypes = [i32, vp, vp, vp, vp, i64, i32, i32, vp]
         lib.bcnn_auto_engine.argtypes = [i32] * 10
@@ -146,6 +152,37 @@ def bcnn_conv2d_b1_module(x_bits, w_bits, bn_scale, bn_shift, identity, prelu_sl
                                         _p(prelu_slope), _p(next_bias), _p(y_real), _p(y_bits), B, H, W, C_in, C_out,
                                         kh, kw, stride, pad, _stream()), "bcnn_conv2d_b1_module")
     return y_real, y_bits
+
+
+def bcnn_conv2d_b1_branches(x_bits, w_bits, bn_scale, bn_shift, pad_dot, identity, prelu_slope, next_bias, y_real, y_bits,
+                            B, H, W, C_in, C_out, P, kh=1, kw=1):
+    """Module with P parallel binary branches (kh*kw > 1: the P = kh*kw shifted taps of a binary kh x kw convolution)."""
+    _check(load().bcnn_conv2d_b1_branches(_p(x_bits), _p(w_bits), _p(bn_scale), _p(bn_shift), _p(pad_dot), _p(identity),
+                                          _p(prelu_slope), _p(next_bias), _p(y_real), _p(y_bits), B, H, W, C_in, C_out, P,
+                                          kh, kw, _stream()), "bcnn_conv2d_b1_branches")
+    return y_real, y_bits
+
+
+def bcnn_dwconv3x3_module(x, w, bn_scale, bn_shift, prelu_slope, next_bias, y_real, y_bits, B, H, W, C_in, R=1, S=1):
+    """Real depth-wise 3x3 convolution (stride S, replication R) -> batch norm -> PReLU -> fp16 map (+ next signs)."""
+    _check(load().bcnn_dwconv3x3_module(_p(x), _p(w), _p(bn_scale), _p(bn_shift), _p(prelu_slope), _p(next_bias), _p(y_real),
+                                        _p(y_bits), B, H, W, C_in, R, S, _stream()), "bcnn_dwconv3x3_module")
+    return y_real, y_bits
+
+
+def bcnn_avgpool(x, y, B, H, W, C_in, R=1, S=1):
+    _check(load().bcnn_avgpool(_p(x), _p(y), B, H, W, C_in, R, S, _stream()), "bcnn_avgpool")
+    return y
+
+
+def bcnn_gap(x, pooled, B, H, W, C):
+    _check(load().bcnn_gap(_p(x), _p(pooled), B, H, W, C, _stream()), "bcnn_gap")
+    return pooled
+
+
+def bcnn_fc(pooled, w, bias, logits, B, C, N):
+    _check(load().bcnn_fc(_p(pooled), _p(w), _p(bias), _p(logits), B, C, N, _stream()), "bcnn_fc")
+    return logits
 
 
 def bcnn_auto_engine(B, H, W, C_in, C_out, kh, kw, stride, pad, fused=True) -> str:

@@ -218,6 +218,80 @@ int bcnn_conv2d_b1_module(const void *x_bits, const void *w_bits, const float *b
     return launch_conv_tc_i8(p, static_cast<cudaStream_t>(stream));
 }
 
+int bcnn_conv2d_b1_branches(const void *x_bits, const void *w_bits, const float *bn_scale, const float *bn_shift,
+                            const int32_t *pad_dot, const void *identity, const float *prelu_slope, const float *next_bias,
+                            void *y_real, void *y_bits, int B, int H, int W, int C_in, int C_out, int P, int kh, int kw,
+                            void *stream)
+{
+    if (!x_bits || !w_bits || !bn_scale || !bn_shift || !prelu_slope || !y_real) return BCNN_ERR_INVALID_ARG;
+    if (B <= 0 || H <= 0 || W <= 0 || C_in <= 0 || C_out <= 0 || P <= 0 || kh <= 0 || kw <= 0) return BCNN_ERR_INVALID_ARG;
+    if (kh * kw > 1 && P != kh * kw) return BCNN_ERR_INVALID_ARG;
+    if (C_in % 32 != 0 || C_out % 32 != 0 || P > 64 || (kh % 2 == 0) || (kw % 2 == 0)) return BCNN_ERR_UNSUPPORTED;
+    if (!aligned16(x_bits) || !aligned16(w_bits) || !aligned16(bn_scale) || !aligned16(bn_shift) || !aligned16(prelu_slope) ||
+        !aligned16(y_real) || (pad_dot && !aligned16(pad_dot)) || (identity && !aligned16(identity)) ||
+        (next_bias && !aligned16(next_bias)) || (y_bits && !aligned16(y_bits)))
+        return BCNN_ERR_ALIGNMENT;
+    BranchProblem p;
+    p.x = static_cast<const uint32_t *>(x_bits);
+    p.w = static_cast<const uint32_t *>(w_bits);
+    p.bn_scale = bn_scale; p.bn_shift = bn_shift; p.pad_dot = pad_dot;
+    p.identity = static_cast<const uint16_t *>(identity);
+    p.slope = prelu_slope; p.next_bias = next_bias;
+    p.y_real = static_cast<uint16_t *>(y_real);
+    p.y_bits = static_cast<uint8_t *>(y_bits);
+    p.B = B; p.H = H; p.W = W; p.C_in = C_in; p.C_out = C_out; p.P = P; p.kh = kh; p.kw = kw;
+    p.cw = C_in / 32;
+    p.M = (long)B * H * W;
+    if (p.M >= (1L << 40)) return BCNN_ERR_UNSUPPORTED;
+    return launch_conv_branches(p, static_cast<cudaStream_t>(stream));
+}
+
+int bcnn_dwconv3x3_module(const void *x, const float *w, const float *bn_scale, const float *bn_shift, const float *prelu_slope,
+                          const float *next_bias, void *y_real, void *y_bits, int B, int H, int W, int C_in, int R, int S,
+                          void *stream)
+{
+    if (!x || !w || !bn_scale || !bn_shift || !prelu_slope || !y_real) return BCNN_ERR_INVALID_ARG;
+    if (B <= 0 || H <= 0 || W <= 0 || C_in <= 0 || R <= 0 || S <= 0) return BCNN_ERR_INVALID_ARG;
+    const long C = (long)C_in * R;
+    if (C_in % 8 != 0 || C >= (1L << 20) || (y_bits && C % 32 != 0)) return BCNN_ERR_UNSUPPORTED;
+    if (!aligned16(x) || !aligned16(w) || !aligned16(bn_scale) || !aligned16(bn_shift) || !aligned16(prelu_slope) ||
+        !aligned16(y_real) || (next_bias && !aligned16(next_bias)) || (y_bits && !aligned16(y_bits)))
+        return BCNN_ERR_ALIGNMENT;
+    if ((long)B * H * W * C >= (1L << 46)) return BCNN_ERR_UNSUPPORTED;
+    return launch_dwconv3x3_module(static_cast<const uint16_t *>(x), w, bn_scale, bn_shift, prelu_slope, next_bias,
+                                   static_cast<uint16_t *>(y_real), static_cast<uint8_t *>(y_bits), B, H, W, C_in, R, S,
+                                   static_cast<cudaStream_t>(stream));
+}
+
+int bcnn_avgpool(const void *x, void *y, int B, int H, int W, int C_in, int R, int S, void *stream)
+{
+    if (!x || !y) return BCNN_ERR_INVALID_ARG;
+    if (B <= 0 || H <= 0 || W <= 0 || C_in <= 0 || R <= 0 || S <= 0) return BCNN_ERR_INVALID_ARG;
+    if (H % S != 0 || W % S != 0) return BCNN_ERR_INVALID_ARG;
+    if (C_in % 8 != 0 || (long)C_in * R >= (1L << 20) || (long)B * H * W * C_in * R >= (1L << 46)) return BCNN_ERR_UNSUPPORTED;
+    if (!aligned16(x) || !aligned16(y)) return BCNN_ERR_ALIGNMENT;
+    return launch_avgpool(static_cast<const uint16_t *>(x), static_cast<uint16_t *>(y), B, H, W, C_in, R, S,
+                          static_cast<cudaStream_t>(stream));
+}
+
+int bcnn_gap(const void *x, float *pooled, int B, int H, int W, int C, void *stream)
+{
+    if (!x || !pooled) return BCNN_ERR_INVALID_ARG;
+    if (B <= 0 || H <= 0 || W <= 0 || C <= 0) return BCNN_ERR_INVALID_ARG;
+    if (C % 8 != 0 || (long)H * W >= (1L << 24) || (long)B * H * W * C >= (1L << 46)) return BCNN_ERR_UNSUPPORTED;
+    if (!aligned16(x) || !aligned16(pooled)) return BCNN_ERR_ALIGNMENT;
+    return launch_gap(static_cast<const uint16_t *>(x), pooled, B, H * W, C, static_cast<cudaStream_t>(stream));
+}
+
+int bcnn_fc(const float *pooled, const float *w, const float *bias, float *logits, int B, int C, int N, void *stream)
+{
+    if (!pooled || !w || !logits) return BCNN_ERR_INVALID_ARG;
+    if (B <= 0 || C <= 0 || N <= 0) return BCNN_ERR_INVALID_ARG;
+    if (C % 4 != 0) return BCNN_ERR_UNSUPPORTED;
+    if (!aligned16(pooled) || !aligned16(w) || !aligned16(logits) || (bias && !aligned16(bias))) return BCNN_ERR_ALIGNMENT;
+    return launch_fc(pooled, w, bias, logits, B, C, N, static_cast<cudaStream_t>(stream));
+}
+
 int bcnn_conv2d_b1_engine(int engine, const void *x_bits, const void *w_bits, const int32_t *thr, void *out,
                           int B, int H, int W, int C_in, int C_out, int kh, int kw, int stride, int pad,
                           void *stream)

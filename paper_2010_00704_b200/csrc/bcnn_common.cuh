@@ -31,6 +31,21 @@ struct ConvProblem {
     uint32_t ohw_mul, ohw_shift;  // exact division of any 32-bit value by OH * OW
 };
 
+// Convolution module with P parallel binary branches (optionally shifted: P = kh * kw taps of an F x F convolution).
+struct BranchProblem {
+    const uint32_t *x;       // packed [B][H][W][P * C_in]: the P binarizations of the module's real input side by side
+    const uint32_t *w;       // packed [P][C_out][C_in]
+    const float *bn_scale, *bn_shift;   // [P][C_out]
+    const int32_t *pad_dot;  // [P][C_out] or nullptr (0): a branch's result where its shifted pixel lies outside the image
+    const uint16_t *identity;           // fp16 [M][C_out] or nullptr
+    const float *slope, *next_bias;     // [C_out]; next_bias may be nullptr (0)
+    uint16_t *y_real;        // fp16 [M][C_out]
+    uint8_t *y_bits;         // packed [M][C_out / 8] or nullptr
+    int B, H, W, C_in, C_out, P, kh, kw;
+    int cw;                  // C_in / 32
+    long M;                  // B * H * W
+};
+
 // Exact n / d for every 32-bit n with a precomputed (mul, shift) pair: with s = ceil(log2 d) and
 // mul = floor(2^32 * (2^s - d) / d) + 1,  n / d = (t + ((n - t) >> 1)) >> (s - 1),  t = umulhi(n, mul).
 // d == 1 is encoded as shift == 0.
@@ -82,6 +97,13 @@ bool conv_tc_pw_supports(const ConvProblem &p);
 int launch_conv_tc_i8(const ConvProblem &p, cudaStream_t stream);
 bool conv_tc_i8_supports(const ConvProblem &p);
 int launch_selftest_wait_timeout(int polls, cudaStream_t stream);
+int launch_conv_branches(const BranchProblem &p, cudaStream_t stream);
+int launch_dwconv3x3_module(const uint16_t *x, const float *w, const float *scale, const float *shift, const float *slope,
+                            const float *next_bias, uint16_t *y, uint8_t *y_bits, int B, int H, int W, int C_in, int R, int S,
+                            cudaStream_t stream);
+int launch_avgpool(const uint16_t *x, uint16_t *y, int B, int H, int W, int C_in, int R, int S, cudaStream_t stream);
+int launch_gap(const uint16_t *x, float *pooled, int B, int HW, int C, cudaStream_t stream);
+int launch_fc(const float *pooled, const float *w, const float *bias, float *logits, int B, int C, int N, cudaStream_t stream);
 int *device_error_word();   // device address of the error word of the current device (nullptr on failure)
 
 }  // namespace bcnn
