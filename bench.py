@@ -706,11 +706,16 @@ def run_paper1x1(args):
     B, P = args.batch, args.branches
     module = args.epilogue == "module"
     peaks = load_peaks()
-    convs = wl.paper_binary_1x1_convs(P)
+    # with the module epilogue the P branches of a module are ONE call (bcnn_conv2d_b1_branches: P binarizations side
+    # by side in the packed input, P weight sets, P batch norms, summed before the identity); with the threshold
+    # epilogue they are P independent convolutions
+    branch_call = module and P > 1
+    convs = wl.paper_binary_1x1_convs(1 if branch_call else P)
+    PB = P if branch_call else 1
     jobs = []
     for li, (l, count) in enumerate(convs):
         rng = synth.rng_for(6, li)
-        x = torch.from_numpy(synth.random_bits(rng, (l.in_bytes(B),))).cuda()
+        x = torch.from_numpy(synth.random_bits(rng, (PB * l.in_bytes(B),))).cuda()
         ident = yreal = None
         if module:
             # the module's real input (fp16 NHWC, standard normal) and its real output, shared by the repeats
@@ -718,13 +723,14 @@ def run_paper1x1(args):
                                 generator=torch.Generator(device="cuda").manual_seed(synth.seed_for(6, li)))
             yreal = torch.empty(l.M(B) * l.C_out, dtype=torch.float16, device="cuda")
         for c in range(count):
-            Wb = torch.from_numpy(synth.random_bits(rng, (l.w_bytes(),))).cuda()
+            Wb = torch.from_numpy(synth.random_bits(rng, (PB * l.w_bytes(),))).cuda()
             thr = torch.from_numpy(synth.thresholds(rng, l.K, l.C_out)).cuda()
             out = torch.empty(l.out_bits_bytes(B), dtype=torch.uint8, device="cuda")
             extra = None
             if module:
-                sc = torch.from_numpy((rng.standard_normal(l.C_out) / np.sqrt(l.K)).astype(np.float32)).cuda()
-                sh, nb = (torch.from_numpy(synth.real_input(rng, (l.C_out,))).cuda() for _ in range(2))
+                sc = torch.from_numpy((rng.standard_normal(PB * l.C_out) / np.sqrt(l.K)).astype(np.float32)).cuda()
+                sh = torch.from_numpy(synth.real_input(rng, (PB * l.C_out,))).cuda()
+                nb = torch.from_numpy(synth.real_input(rng, (l.C_out,))).cuda()
                 sl = torch.from_numpy(rng.uniform(0.0, 0.5, l.C_out).astype(np.float32)).cuda()
                 extra = (sc, sh, ident, sl, nb, yreal)
             jobs.append((l, x, Wb, thr, out, extra))
@@ -733,7 +739,10 @@ def run_paper1x1(args):
         l, x, Wb, thr, out, extra = j
         if module:
             sc, sh, idn, sl, nb, yr = extra
-            binding.bcnn_conv2d_b1_module(x, Wb, sc, sh, idn, sl, nb, yr, out, B, l.H, l.W, l.C_in, l.C_out, 1, 1, 1, 0)
+            if branch_call:
+                binding.bcnn_conv2d_b1_branches(x, Wb, sc, sh, None, idn, sl, nb, yr, out, B, l.H, l.W, l.C_in, l.C_out, P)
+            else:
+                binding.bcnn_conv2d_b1_module(x, Wb, sc, sh, idn, sl, nb, yr, out, B, l.H, l.W, l.C_in, l.C_out, 1, 1, 1, 0)
         else:
             binding.bcnn_conv2d_b1_fused(x, Wb, thr, out, B, l.H, l.W, l.C_in, l.C_out, 1, 1, 1, 0)
 
@@ -774,14 +783,14 @@ def run_paper1x1(args):
     for l, count in convs:
         ms = float(np.mean([a.elapsed_time(b) for a, b in per[l.name]]))
         shapes.append({"layer": l.name, "count": count, "M": l.M(B), "N": l.C_out, "K": l.K,
-                       "engine": "tc_ws" if module
+                       "engine": ("branches (CUDA cores)" if branch_call else "tc_ws") if module
                        else binding.bcnn_auto_engine(B, l.H, l.W, l.C_in, l.C_out, 1, 1, 1, 0),
-                       "ms_per_launch": ms, "tops": l.ops(B) / (ms / 1e3) / 1e12})
+                       "ms_per_launch": ms, "tops": PB * l.ops(B) / (ms / 1e3) / 1e12})
         # algorithmic bytes: packed input + packed output (+ fp16 identity read and fp16 map written by the module)
-        nbytes = l.in_bytes(B) + l.out_bits_bytes(B) + (4 * l.M(B) * l.C_out if module else 0)
+        nbytes = PB * l.in_bytes(B) + l.out_bits_bytes(B) + (4 * l.M(B) * l.C_out if module else 0)
         shapes[-1].update({"gbs": nbytes / (ms / 1e3) / 1e9, "hbm_frac": nbytes / (ms / 1e3) / 1e9 / peaks["hbm_gbs"]})
     err = binding.bcnn_device_error()
-    ops = 2 * sum(n * l.macs(B) for l, n in convs)
+    ops = 2 * PB * sum(n * l.macs(B) for l, n in convs)
     print(json.dumps({
         "mode": "paper1x1", "epilogue": args.epilogue, "metric": "binary conv throughput (2*M*N*K bit-ops/s), the paper's 1x1 convolutions (Table 1)",
         "value": ops / (ms_step / 1e3) / 1e12, "unit": UNIT, "ms_per_step": ms_step, "images_per_s": B / (ms_step / 1e3),
@@ -794,9 +803,64 @@ def run_paper1x1(args):
     return 0 if err == 0 else 1
 
 
+def run_block(args):
+    """The real-valued vector operations of the paper's building block and head at the shapes of Table 1 (not the
+    headline line): depth-wise 3x3 module at stride 1 and 2 (with the next module's sign bits), S x S average pooling
+    with replication on the identity path, global pooling + fully connected layer; median of --steps launches with L2
+    flushed in between; achieved GB/s on algorithmic bytes against the measured copy bandwidth.  One JSON line."""
+    import torch
+    from paper_2010_00704_b200 import build, binding
+    build.build()
+    binding.load()
+    torch.cuda.set_device(0)
+    B = args.batch
+    peaks = load_peaks()
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    gen = torch.Generator(device="cuda").manual_seed(synth.seed_for(7))
+    rows = []
+
+    def add(name, fn, nbytes):
+        ts = timed_launches(fn, args.steps, args.warmup, flush)
+        med = float(np.median(ts))
+        rows.append({"op": name, "ms_median": med, "ms_min": float(min(ts)), "algorithmic_bytes": int(nbytes),
+                     "gbs": nbytes / (med / 1e3) / 1e9, "hbm_frac": nbytes / (med / 1e3) / 1e9 / peaks["hbm_gbs"]})
+
+    def f32(n):
+        return torch.randn(n, dtype=torch.float32, device="cuda", generator=gen)
+
+    # (level, resolution of the block's input, channels before replication, R, S) of the down-sampling blocks and of
+    # one normal block per level (Table 1)
+    for name, H, C_in, R, S in (("level1 down", 224, 32, 2, 2), ("level2 down", 112, 64, 2, 2), ("level3 down", 56, 128, 2, 2),
+                                ("level3 normal", 28, 256, 1, 1), ("level4 down", 28, 256, 2, 2), ("level4 normal", 14, 512, 1, 1),
+                                ("level5 down", 14, 512, 2, 2), ("level5 normal", 7, 1024, 1, 1)):
+        C = C_in * R
+        OH = (H - 1) // S + 1
+        x = torch.randn(B * H * H * C_in, dtype=torch.float16, device="cuda", generator=gen)
+        y = torch.empty(B * OH * OH * C, dtype=torch.float16, device="cuda")
+        bits = torch.empty(B * OH * OH * C // 8, dtype=torch.uint8, device="cuda")
+        w, sc, sh, sl, nb = f32(C * 9), f32(C), f32(C), f32(C), f32(C)
+        add(f"{name}: depth-wise 3x3 / {S} module {H}x{H}x{C_in} -> {OH}x{OH}x{C} (+ next signs)",
+            lambda: binding.bcnn_dwconv3x3_module(x, w, sc, sh, sl, nb, y, bits, B, H, H, C_in, R, S),
+            2 * x.numel() + 2 * y.numel() + bits.numel())
+        if S > 1:
+            add(f"{name}: {S}x{S}/{S} average pooling, replication {R}, {H}x{H}x{C_in} -> {OH}x{OH}x{C}",
+                lambda: binding.bcnn_avgpool(x, y, B, H, H, C_in, R, S), 2 * x.numel() + 2 * y.numel())
+        del x, y, bits
+    x = torch.randn(B * 49 * 1024, dtype=torch.float16, device="cuda", generator=gen)
+    pooled = torch.empty(B * 1024, dtype=torch.float32, device="cuda")
+    logits = torch.empty(B * 1000, dtype=torch.float32, device="cuda")
+    wfc, bfc = f32(1000 * 1024), f32(1000)
+    add("head: global average pooling 7x7x1024", lambda: binding.bcnn_gap(x, pooled, B, 7, 7, 1024), 2 * x.numel() + 4 * pooled.numel())
+    add("head: fully connected 1024 -> 1000", lambda: binding.bcnn_fc(pooled, wfc, bfc, logits, B, 1024, 1000),
+        4 * (pooled.numel() + wfc.numel() + logits.numel()))
+    print(json.dumps({"mode": "block", "batch": B, "hbm_peak_gbs": peaks["hbm_gbs"], "peak_source": peaks["source"], "ops": rows,
+                      "device_error": binding.bcnn_device_error()}))
+    return 0
+
+
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("--mode", default="bench", choices=["bench", "sweep", "paper1x1"])
+    ap.add_argument("--mode", default="bench", choices=["bench", "sweep", "paper1x1", "block"])
     ap.add_argument("--engines", default="auto,lop3,mma_b1,tc_i8,mma_s8,tc_ws,tc_pw")
     ap.add_argument("--sweep-set", default="all", choices=["gemm", "conv", "all"])
     ap.add_argument("--only", default="", help="sweep mode: run only shapes whose label contains this text")
@@ -819,6 +883,8 @@ def main():
         return run_sweep(args)
     if args.mode == "paper1x1":
         return run_paper1x1(args)
+    if args.mode == "block":
+        return run_block(args)
     return run_gpu(args)
 
 
