@@ -657,9 +657,13 @@ def run_sweep(args):
             outb = torch.empty(M * N // 8, dtype=torch.uint8, device="cuda")
             ops = wl.gemm_ops(M, N, K)
             name = f"gemm M=N={M} K={K}"
+            prep = torch.empty(binding.bcnn_prepared_weights_bytes(N, K), dtype=torch.uint8, device="cuda")
+            binding.bcnn_prepare_weights(Wb, prep, N, K)
             calls = {
-                "int32": lambda e: binding.bcnn_gemm_b1(A, Wb, out32, M, N, K, engine=e),
-                "fused": lambda e: binding.bcnn_gemm_b1_fused(A, Wb, thr, outb, M, N, K, engine=e),
+                "int32": lambda e: binding.bcnn_gemm_b1_prepared(A, prep, None, out32, M, N, K) if e == "tc_pre"
+                else binding.bcnn_gemm_b1(A, Wb, out32, M, N, K, engine=e),
+                "fused": lambda e: binding.bcnn_gemm_b1_prepared(A, prep, thr, outb, M, N, K) if e == "tc_pre"
+                else binding.bcnn_gemm_b1_fused(A, Wb, thr, outb, M, N, K, engine=e),
             }
             out_bytes = {"int32": 4 * M * N, "fused": M * N // 8}
         else:
@@ -669,16 +673,20 @@ def run_sweep(args):
             outb = torch.empty(l.out_bits_bytes(B), dtype=torch.uint8, device="cuda")
             ops = l.ops(B)
             name = f"conv {l.name} B={B} M={l.M(B)} N={l.C_out} K={l.K}"
+            prep = torch.empty(binding.bcnn_prepared_weights_bytes(l.C_out, l.K), dtype=torch.uint8, device="cuda")
+            binding.bcnn_prepare_weights(Wb, prep, l.C_out, l.K)
             calls = {
-                "fused": lambda e: binding.bcnn_conv2d_b1_fused(x, Wb, thr, outb, B, l.H, l.W, l.C_in, l.C_out,
-                                                                 l.k, l.k, l.stride, l.pad, engine=e),
+                "fused": lambda e: binding.bcnn_conv2d_b1_prepared(x, prep, thr, outb, B, l.H, l.W, l.C_in, l.C_out, l.k, l.k,
+                                                                    l.stride, l.pad) if e == "tc_pre"
+                else binding.bcnn_conv2d_b1_fused(x, Wb, thr, outb, B, l.H, l.W, l.C_in, l.C_out,
+                                                  l.k, l.k, l.stride, l.pad, engine=e),
             }
             out_bytes = {"fused": l.out_bits_bytes(B)}
         for okind, call in calls.items():
             if okind not in args.outs.split(","):
                 continue
             for en in engines:
-                e = binding.ENGINES[en]
+                e = "tc_pre" if en == "tc_pre" else binding.ENGINES[en]      # tc_pre: the *_prepared calls (weights expanded once)
                 try:
                     med, mn_ = timeit(lambda: call(e))
                 except binding.BcnnError as ex:
@@ -861,7 +869,7 @@ def run_block(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--mode", default="bench", choices=["bench", "sweep", "paper1x1", "block"])
-    ap.add_argument("--engines", default="auto,lop3,mma_b1,tc_i8,mma_s8,tc_ws,tc_pw")
+    ap.add_argument("--engines", default="auto,lop3,mma_b1,tc_i8,mma_s8,tc_ws,tc_pw,tc_pre")
     ap.add_argument("--sweep-set", default="all", choices=["gemm", "conv", "all"])
     ap.add_argument("--only", default="", help="sweep mode: run only shapes whose label contains this text")
     ap.add_argument("--outs", default="int32,fused", help="sweep mode: output kinds to run")

@@ -220,6 +220,28 @@ int bcnn_gemm_b1_engine(int engine, const void *A_bits, const void *W_bits, cons
                         void *out, int64_t M, int N, int K, void *stream);
 
 /*
+ * Prepared weights.  A layer's weights do not change between calls; expanding their sign bits to the signed bytes the
+ * tensor cores multiply is done once, into a buffer the CALLER owns (the library never allocates), and the *_prepared
+ * calls then stream that buffer by TMA instead of expanding the weight bits again for every tile of every call.
+ * Worth it for wide layers and long K (C_out > 128: bcnn_prepared_preferred tells); results are bit-identical to the
+ * plain calls.
+ *   bcnn_prepared_weights_bytes(C_out, K)   size of the buffer for C_out rows of K = kh*kw*C_in bits (0 if invalid)
+ *   bcnn_prepare_weights(w_bits, prepared, C_out, K, stream)   w_bits as in bcnn_conv2d_b1; prepared: device, 256-byte
+ *                                           aligned, at least that many bytes; enqueues one small kernel
+ *   bcnn_conv2d_b1_prepared / bcnn_gemm_b1_prepared   as bcnn_conv2d_b1_engine / bcnn_gemm_b1_engine with `prepared` in
+ *                                           place of w_bits: thr == NULL selects the int32 output, else packed bits
+ *   bcnn_prepared_preferred(...)            1 if the prepared call is expected to be the faster one for this shape
+ * BCNN_ERR_UNSUPPORTED for shapes the engine does not take (the caller then uses the plain call).
+ */
+size_t bcnn_prepared_weights_bytes(int C_out, int K);
+int bcnn_prepare_weights(const void *w_bits, void *prepared, int C_out, int K, void *stream);
+int bcnn_conv2d_b1_prepared(const void *x_bits, const void *prepared, const int32_t *thr, void *out,
+                            int B, int H, int W, int C_in, int C_out, int kh, int kw, int stride, int pad, void *stream);
+int bcnn_gemm_b1_prepared(const void *A_bits, const void *prepared, const int32_t *thr, void *out,
+                          int64_t M, int N, int K, void *stream);
+int bcnn_prepared_preferred(int B, int H, int W, int C_in, int C_out, int kh, int kw, int stride, int pad, int fused);
+
+/*
  * Which engine BCNN_ENGINE_AUTO runs for a convolution of this shape (fused != 0: the packed
  * output).  Returns a bcnn_engine value, or a negative bcnn_status for an invalid shape.
  * No pointers, no launch.  A GEMM is the shape (1, M, 1, K, N, 1, 1, 1, 0).

@@ -22,6 +22,7 @@ ENGINES = {"auto": ENGINE_AUTO, "lop3": ENGINE_LOP3, "mma_b1": ENGINE_MMA_B1, "t
 EXPORTS = (
     "bcnn_pack", "bcnn_stem_fused", "bcnn_gemm_b1", "bcnn_gemm_b1_fused", "bcnn_conv2d_b1", "bcnn_conv2d_b1_fused", "bcnn_conv2d_b1_module",
     "bcnn_conv2d_b1_branches", "bcnn_dwconv3x3_module", "bcnn_avgpool", "bcnn_gap", "bcnn_fc",
+    "bcnn_prepared_weights_bytes", "bcnn_prepare_weights", "bcnn_conv2d_b1_prepared", "bcnn_gemm_b1_prepared", "bcnn_prepared_preferred",
     "bcnn_conv2d_b1_engine", "bcnn_gemm_b1_engine", "bcnn_auto_engine", "bcnn_device_error", "bcnn_device_status",
     "bcnn_workspace_bytes", "bcnn_selftest_wait_timeout", "bcnn_status_string", "bcnn_version",
 )
@@ -59,6 +60,12 @@ def load() -> ctypes.CDLL:
         lib.bcnn_avgpool.argtypes = [vp, vp] + [i32] * 6 + [vp]
         lib.bcnn_gap.argtypes = [vp, vp] + [i32] * 4 + [vp]
         lib.bcnn_fc.argtypes = [vp] * 4 + [i32] * 3 + [vp]
+        lib.bcnn_prepared_weights_bytes.argtypes = [i32, i32]
+        lib.bcnn_prepared_weights_bytes.restype = ctypes.c_size_t
+        lib.bcnn_prepare_weights.argtypes = [vp, vp, i32, i32, vp]
+        lib.bcnn_conv2d_b1_prepared.argtypes = [vp, vp, vp, vp] + [i32] * 9 + [vp]
+        lib.bcnn_gemm_b1_prepared.argtypes = [vp, vp, vp, vp, i64, i32, i32, vp]
+        lib.bcnn_prepared_preferred.argtypes = [i32] * 10
         lib.bcnn_conv2d_b1_engine.argtypes = [i32, vp, vp, vp, vp] + [i32] * 9 + [vp]
         lib.bcnn_gemm_b1_engine.argtypes = [i32, vp, vp, vp, vp, i64, i32, i32, vp]
         lib.bcnn_auto_engine.argtypes = [i32] * 10
@@ -70,7 +77,7 @@ def load() -> ctypes.CDLL:
         lib.bcnn_status_string.argtypes = [i32]
         lib.bcnn_status_string.restype = ctypes.c_char_p
         for name in EXPORTS:
-            if name not in ("bcnn_status_string", "bcnn_workspace_bytes"):
+            if name not in ("bcnn_status_string", "bcnn_workspace_bytes", "bcnn_prepared_weights_bytes"):
                 getattr(lib, name).restype = i32
         _lib = lib
     return _lib
@@ -183,6 +190,31 @@ def bcnn_gap(x, pooled, B, H, W, C):
 def bcnn_fc(pooled, w, bias, logits, B, C, N):
     _check(load().bcnn_fc(_p(pooled), _p(w), _p(bias), _p(logits), B, C, N, _stream()), "bcnn_fc")
     return logits
+
+
+def bcnn_prepared_weights_bytes(C_out, K) -> int:
+    return int(load().bcnn_prepared_weights_bytes(C_out, K))
+
+
+def bcnn_prepare_weights(w_bits, prepared, C_out, K):
+    """Expand a layer's packed weights once into the caller's buffer ``prepared`` (256-byte aligned)."""
+    _check(load().bcnn_prepare_weights(_p(w_bits), _p(prepared), C_out, K, _stream()), "bcnn_prepare_weights")
+    return prepared
+
+
+def bcnn_conv2d_b1_prepared(x_bits, prepared, thr, out, B, H, W, C_in, C_out, kh, kw, stride, pad):
+    _check(load().bcnn_conv2d_b1_prepared(_p(x_bits), _p(prepared), _p(thr), _p(out), B, H, W, C_in, C_out, kh, kw, stride, pad,
+                                          _stream()), "bcnn_conv2d_b1_prepared")
+    return out
+
+
+def bcnn_gemm_b1_prepared(A_bits, prepared, thr, out, M, N, K):
+    _check(load().bcnn_gemm_b1_prepared(_p(A_bits), _p(prepared), _p(thr), _p(out), M, N, K, _stream()), "bcnn_gemm_b1_prepared")
+    return out
+
+
+def bcnn_prepared_preferred(B, H, W, C_in, C_out, kh, kw, stride, pad, fused=True) -> bool:
+    return bool(load().bcnn_prepared_preferred(B, H, W, C_in, C_out, kh, kw, stride, pad, 1 if fused else 0))
 
 
 def bcnn_auto_engine(B, H, W, C_in, C_out, kh, kw, stride, pad, fused=True) -> str:

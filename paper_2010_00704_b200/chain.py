@@ -18,13 +18,15 @@ from .workloads import ConvLayer
 class FusedChain:
     def __init__(self, layers, batch: int, w_bits_list, thr_list, real_input_shape=None, bias=None,
                  replicate: int = 1, engine: int = binding.ENGINE_AUTO, keep_all: bool = False,
-                 device="cuda", fuse_stem=None):
+                 device="cuda", fuse_stem=None, prepare_weights=None):
         """layers: sequence of ConvLayer; w_bits_list[i]: uint8 numpy [C_out, k, k, C_in/8];
         thr_list[i]: int32 numpy [C_out].  real_input_shape = (H, W, C_real) enables the pack
         stage (fp32 NHWC input, optional per-channel bias, replication factor).
         keep_all keeps one output buffer per layer (for checking) instead of two ping-pong buffers.
         fuse_stem: run pack + first layer as one ``bcnn_stem_fused`` call (the packed input is then never
-        written); default: whenever the shapes allow it and keep_all is off."""
+        written); default: whenever the shapes allow it and keep_all is off.
+        prepare_weights: expand the weights of wide / long-K layers once (``bcnn_prepare_weights``) and run those layers
+        through ``bcnn_conv2d_b1_prepared``; default: with the AUTO engine."""
         self.layers = list(layers)
         self.batch = int(batch)
         self.engine = engine
@@ -57,6 +59,18 @@ class FusedChain:
         if self.fuse_stem and not can_fuse:
             raise ValueError("fuse_stem needs a 4-channel real input replicated 8x and a first 1x1 layer 32 -> 32")
         self.launches_per_run = len(self.layers) + (1 if real_input_shape is not None and not self.fuse_stem else 0)
+        # wide layers / long K: the layer's weights are expanded once, here, into a buffer this object owns, and the
+        # *_prepared call streams them by TMA (bit-identical results); everything else takes the plain fused call
+        self.prepared = [None] * len(self.layers)
+        if prepare_weights is None:
+            prepare_weights = engine == binding.ENGINE_AUTO
+        if prepare_weights:
+            for i, l in enumerate(self.layers):
+                if binding.bcnn_prepared_preferred(self.batch, l.H, l.W, l.C_in, l.C_out, l.k, l.k, l.stride, l.pad):
+                    buf = torch.empty(binding.bcnn_prepared_weights_bytes(l.C_out, l.K), dtype=torch.uint8, device=self.device)
+                    binding.bcnn_prepare_weights(self.w[i], buf, l.C_out, l.K)
+                    self.prepared[i] = buf
+            torch.cuda.synchronize()
 
     def enqueue_pack(self, x_real):
         H, W, C = self.real_input_shape
@@ -75,8 +89,12 @@ class FusedChain:
             if i == 0 and self.fuse_stem:        # done by enqueue_pack
                 cur = o
                 continue
-            binding.bcnn_conv2d_b1_fused(cur, w, t, o, self.batch, l.H, l.W, l.C_in, l.C_out, l.k, l.k,
-                                         l.stride, l.pad, engine=self.engine)
+            if self.prepared[i] is not None:
+                binding.bcnn_conv2d_b1_prepared(cur, self.prepared[i], t, o, self.batch, l.H, l.W, l.C_in, l.C_out, l.k, l.k,
+                                                l.stride, l.pad)
+            else:
+                binding.bcnn_conv2d_b1_fused(cur, w, t, o, self.batch, l.H, l.W, l.C_in, l.C_out, l.k, l.k,
+                                             l.stride, l.pad, engine=self.engine)
             cur = o
         return cur
 

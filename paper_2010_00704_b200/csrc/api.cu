@@ -312,6 +312,56 @@ int bcnn_gemm_b1_engine(int engine, const void *A_bits, const void *W_bits, cons
     return dispatch(engine, p, static_cast<cudaStream_t>(stream));
 }
 
+size_t bcnn_prepared_weights_bytes(int C_out, int K)
+{
+    if (C_out <= 0 || K <= 0 || K % 32 != 0 || K >= (1 << 30)) return 0;
+    PreparedWeights pw;
+    size_t bytes = 0;
+    prepared_layout(C_out, K, pw, bytes);
+    return bytes;
+}
+
+int bcnn_prepare_weights(const void *w_bits, void *prepared, int C_out, int K, void *stream)
+{
+    if (!w_bits || !prepared || C_out <= 0 || K <= 0) return BCNN_ERR_INVALID_ARG;
+    if (K % 32 != 0 || K >= (1 << 30)) return BCNN_ERR_UNSUPPORTED;
+    if (!aligned16(w_bits) || (reinterpret_cast<uintptr_t>(prepared) & 255u) != 0) return BCNN_ERR_ALIGNMENT;
+    return launch_prepare_weights(static_cast<const uint32_t *>(w_bits), prepared, C_out, K, static_cast<cudaStream_t>(stream));
+}
+
+int bcnn_conv2d_b1_prepared(const void *x_bits, const void *prepared, const int32_t *thr, void *out,
+                            int B, int H, int W, int C_in, int C_out, int kh, int kw, int stride, int pad, void *stream)
+{
+    ConvProblem p;
+    const int st = make_conv_problem(p, x_bits, prepared, thr, out, B, H, W, C_in, C_out, kh, kw, stride, pad, thr != nullptr);
+    if (st != BCNN_OK) return st;
+    if ((reinterpret_cast<uintptr_t>(prepared) & 255u) != 0) return BCNN_ERR_ALIGNMENT;
+    return launch_conv_tc_pre(p, prepared, static_cast<cudaStream_t>(stream));
+}
+
+int bcnn_gemm_b1_prepared(const void *A_bits, const void *prepared, const int32_t *thr, void *out,
+                          int64_t M, int N, int K, void *stream)
+{
+    ConvProblem p;
+    const int st = gemm_problem(p, A_bits, prepared, thr, out, M, N, K, thr != nullptr);
+    if (st != BCNN_OK) return st;
+    if ((reinterpret_cast<uintptr_t>(prepared) & 255u) != 0) return BCNN_ERR_ALIGNMENT;
+    return launch_conv_tc_pre(p, prepared, static_cast<cudaStream_t>(stream));
+}
+
+int bcnn_prepared_preferred(int B, int H, int W, int C_in, int C_out, int kh, int kw, int stride, int pad, int fused)
+{
+    ConvProblem p;
+    void *dummy = reinterpret_cast<void *>(uintptr_t(4096));
+    const int st = make_conv_problem(p, dummy, dummy, fused ? static_cast<const int32_t *>(dummy) : nullptr, dummy,
+                                     B, H, W, C_in, C_out, kh, kw, stride, pad, fused != 0);
+    if (st != BCNN_OK) return 0;
+    // measured (bench.py --mode sweep): streaming prepared weights wins wherever AUTO would run the streaming engine
+    // (wide layers, long K) and on every K >= 2048; the weight-stationary and pointwise engines keep the short-K layers
+    if (!conv_tc_pre_supports(p)) return 0;
+    return (auto_engine(p) == BCNN_ENGINE_TC_I8 || p.K >= 2048) ? 1 : 0;
+}
+
 int bcnn_auto_engine(int B, int H, int W, int C_in, int C_out, int kh, int kw, int stride, int pad, int fused)
 {
     ConvProblem p;
@@ -376,6 +426,10 @@ const char *bcnn_status_string(int status)
     case 122: return "device wait timed out: pointwise tcgen05 engine, producer waiting for a chunk's rows";
     case 123: return "device wait timed out: pointwise tcgen05 engine, issuer waiting for a slot's expanded rows";
     case 124: return "device wait timed out: pointwise tcgen05 engine, epilogue waiting for a chunk's accumulators";
+    case 131: return "device wait timed out: prepared-weights tcgen05 engine, producer waiting for a free ring slot";
+    case 132: return "device wait timed out: prepared-weights tcgen05 engine, control warp waiting for a full slot or a free accumulator";
+    case 133: return "device wait timed out: prepared-weights tcgen05 engine, epilogue waiting for an accumulator";
+    case 134: return "device wait timed out: prepared-weights tcgen05 engine, loader waiting for a free ring slot";
     case 125: return "device wait timed out: pointwise tcgen05 engine, producer waiting for a slot's previous MMAs";
     case 126: return "device wait timed out: pointwise tcgen05 engine, issuer waiting for a slot's accumulators";
     case BCNN_SELFTEST_TIMEOUT_CODE: return "device wait timed out: self-test (expected)";

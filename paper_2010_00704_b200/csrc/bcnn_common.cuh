@@ -95,6 +95,17 @@ bool conv_tc_ws_supports(const ConvProblem &p);
 int launch_conv_tc_pw(const ConvProblem &p, cudaStream_t stream);
 bool conv_tc_pw_supports(const ConvProblem &p);
 int launch_conv_tc_i8(const ConvProblem &p, cudaStream_t stream);
+// weights expanded once per layer by launch_prepare_weights (conv_tc_pre.cu): [n_pad][k_pad] signed bytes, then
+// K - 2 popc(W_n) per row
+struct PreparedWeights {
+    const uint8_t *wexp;
+    const int32_t *cst;
+    int n_pad, k_pad;
+};
+void prepared_layout(int C_out, int K, PreparedWeights &pw, size_t &bytes);
+int launch_prepare_weights(const uint32_t *w, void *prepared, int C_out, int K, cudaStream_t stream);
+int launch_conv_tc_pre(const ConvProblem &p, const void *prepared, cudaStream_t stream);
+bool conv_tc_pre_supports(const ConvProblem &p);
 bool conv_tc_i8_supports(const ConvProblem &p);
 int launch_selftest_wait_timeout(int polls, cudaStream_t stream);
 int launch_conv_branches(const BranchProblem &p, cudaStream_t stream);

@@ -352,6 +352,96 @@ def test_errors_launch_nothing(bk):
     assert bk.bcnn_device_error() == 0
 
 
+PREPARED_SHAPES = [
+    # B, H, W, Ci, Co, kh, kw, stride, pad
+    (1, 40, 40, 256, 256, 3, 3, 2, 1),     # several M tiles, K = 2304, one 256-wide tile column
+    (5, 14, 14, 512, 64, 3, 3, 1, 1),      # K = 4608, narrow N (128-wide tile, half of it padding)
+    (2, 6, 9, 160, 224, 1, 3, 1, 2),       # ragged N, K = 480 (not a multiple of 128), pad 2
+    (1, 32, 32, 128, 128, 3, 3, 1, 1),     # the single 3x3 workload
+    (2, 9, 13, 32, 64, 3, 3, 1, 1),        # one-word pixels, K = 288
+    (1, 17, 5, 32, 160, 3, 1, 2, 0),       # kh != kw
+    (3, 7, 11, 96, 32, 1, 1, 1, 0),        # 1x1, K = 96
+    (1, 13, 17, 512, 512, 1, 1, 1, 0),     # wide 1x1: two 256-wide tile columns, several M tiles
+]
+
+
+@pytest.mark.parametrize("shape", PREPARED_SHAPES)
+def test_conv_prepared_weights(bk, oracle, shape):
+    # weights expanded once into a caller-owned buffer, then streamed by TMA: int32 and packed outputs against the
+    # oracle, thresholds with ties and out-of-range values, guard bytes around outputs and the prepared buffer
+    B, H, W, Ci, Co, kh, kw, s, p = shape
+    rng = np.random.default_rng(1900 + sum(shape))
+    x = synth.pm1(rng, (B, H, W, Ci))
+    w = synth.pm1(rng, (Co, kh, kw, Ci))
+    want = oracle.conv2d(x, w, s, p)
+    K = kh * kw * Ci
+    OH, OW = bk.out_hw(H, W, kh, kw, s, p)
+    nbytes = bk.bcnn_prepared_weights_bytes(Co, K)
+    assert nbytes >= Co * K
+    raw_p, prep = guard_alloc(nbytes)
+    assert prep.data_ptr() % 256 == 0
+    xb = dev(synth.pack_bits(x))
+    bk.bcnn_prepare_weights(dev(synth.pack_bits(w)), prep, Co, K)
+    n32 = B * OH * OW * Co * 4
+    raw, buf = guard_alloc(n32)
+    bk.bcnn_conv2d_b1_prepared(xb, prep, None, buf, B, H, W, Ci, Co, kh, kw, s, p)
+    torch.cuda.synchronize()
+    check_guards(raw, n32)
+    check_guards(raw_p, nbytes)
+    assert np.array_equal(buf.cpu().numpy().view(np.int32).reshape(B, OH, OW, Co), want)
+    if Co % 32 == 0:
+        thr = synth.thresholds(rng, K, Co)
+        thr[::3] = want.reshape(-1, Co)[0, ::3]
+        thr = plant_extreme_thresholds(thr, K)
+        nb = B * OH * OW * Co // 8
+        raw, bits = guard_alloc(nb)
+        bk.bcnn_conv2d_b1_prepared(xb, prep, dev(thr), bits, B, H, W, Ci, Co, kh, kw, s, p)
+        torch.cuda.synchronize()
+        check_guards(raw, nb)
+        assert np.array_equal(synth.unpack_bits(bits.cpu().numpy().reshape(B, OH, OW, Co // 8)), oracle.threshold(want, thr))
+    assert bk.bcnn_device_error() == 0
+
+
+@pytest.mark.parametrize("shape", [(1024, 1024, 512), (300, 200, 96), (129, 33, 1056), (64, 512, 4608), (1, 32, 32), (2000, 384, 2304)])
+def test_gemm_prepared_weights(bk, oracle, shape):
+    M, N, K = shape
+    rng = np.random.default_rng(2900 + sum(shape))
+    A, Wt = synth.pm1(rng, (M, K)), synth.pm1(rng, (N, K))
+    want = oracle.gemm(A, Wt)
+    prep = torch.empty(bk.bcnn_prepared_weights_bytes(N, K), dtype=torch.uint8, device="cuda")
+    bk.bcnn_prepare_weights(dev(synth.pack_bits(Wt)), prep, N, K)
+    raw, C = guard_alloc(M * N * 4)
+    bk.bcnn_gemm_b1_prepared(dev(synth.pack_bits(A)), prep, None, C, M, N, K)
+    torch.cuda.synchronize()
+    check_guards(raw, M * N * 4)
+    assert np.array_equal(C.cpu().numpy().view(np.int32).reshape(M, N), want)
+    if N % 32 == 0:
+        thr = plant_extreme_thresholds(synth.thresholds(rng, K, N), K)
+        thr[::4] = want[M // 2, ::4]
+        raw, ob = guard_alloc(M * N // 8)
+        bk.bcnn_gemm_b1_prepared(dev(synth.pack_bits(A)), prep, dev(thr), ob, M, N, K)
+        torch.cuda.synchronize()
+        check_guards(raw, M * N // 8)
+        assert np.array_equal(synth.unpack_bits(ob.cpu().numpy().reshape(M, N // 8)), oracle.threshold(want, thr))
+    assert bk.bcnn_device_error() == 0
+
+
+def test_prepared_errors(bk):
+    a = torch.zeros(1 << 16, dtype=torch.uint8, device="cuda")
+    assert bk.bcnn_prepared_weights_bytes(64, 48) == 0                 # K not a multiple of 32
+    with pytest.raises(bk.BcnnError) as e:
+        bk.bcnn_prepare_weights(a, a[16:], 32, 64)                     # buffer not 256-byte aligned
+    assert e.value.status == -3
+    with pytest.raises(bk.BcnnError) as e:
+        bk.bcnn_conv2d_b1_prepared(a, a, a, a, 1, 4, 4, 32, 48, 1, 1, 1, 0)   # packed output needs C_out % 32 == 0
+    assert e.value.status == -2
+    with pytest.raises(bk.BcnnError) as e:
+        bk.bcnn_gemm_b1_prepared(a, None, None, a, 8, 32, 32)
+    assert e.value.status == -1
+    torch.cuda.synchronize()
+    assert int(a.sum()) == 0
+
+
 def test_bounded_wait_runs_out_and_is_reported(bk, oracle):
     # failure detection without a fault: a wait that nothing satisfies gives up after its poll limit, the kernel
     # frees its tensor memory and ends normally, the error word carries the code until it is read, and the context
