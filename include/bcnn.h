@@ -242,6 +242,27 @@ int bcnn_gemm_b1_prepared(const void *A_bits, const void *prepared, const int32_
 int bcnn_prepared_preferred(int B, int H, int W, int C_in, int C_out, int kh, int kw, int stride, int pad, int fused);
 
 /*
+ * bcnn_conv2d_b1_fused for callers that can neither allocate device memory nor pass a buffer for prepared weights
+ * (the paper has no counterpart: this is a property of the library, not of the method).  Think of code that runs
+ * inside a memory plan it does not own - an inference runtime whose arena was sized before this layer existed, a
+ * plug-in that is handed only its input and output tensors - or at a point where an allocation is not allowed or
+ * would synchronise the device.  The call is bcnn_prepare_weights + bcnn_conv2d_b1_prepared with the prepared form
+ * kept in a static device array inside the library: BCNN_STATIC_SCRATCH_BYTES (4 MiB) that every GPU which loads the
+ * library holds until the process ends.  Arguments and result are exactly those of bcnn_conv2d_b1_fused (bit-identical
+ * output; thr must not be NULL); it allocates and frees nothing.
+ *   - BCNN_ERR_WORKSPACE when bcnn_prepared_weights_bytes(C_out, kh*kw*C_in) exceeds BCNN_STATIC_SCRATCH_BYTES
+ *     (e.g. 512 output channels x 4608 bits fit, 1024 x 9216 do not), BCNN_ERR_UNSUPPORTED as for the prepared call.
+ *   - The first call on a device looks up the array's device address; make that first call outside any stream capture.
+ *   - All calls share the one array and each call overwrites all of it that it uses, so nothing needs clearing; but
+ *     two calls that overlap on the GPU (different streams, or the same call from two threads) race on it.  Calls on
+ *     one stream are ordered and safe.
+ */
+#define BCNN_STATIC_SCRATCH_BYTES (4u << 20)
+int bcnn_conv2d_b1_fused_noalloc(const void *x_bits, const void *w_bits, const int32_t *thr, void *y_bits,
+                                 int B, int H, int W, int C_in, int C_out, int kh, int kw, int stride, int pad,
+                                 void *stream);
+
+/*
  * Which engine BCNN_ENGINE_AUTO runs for a convolution of this shape (fused != 0: the packed
  * output).  Returns a bcnn_engine value, or a negative bcnn_status for an invalid shape.
  * No pointers, no launch.  A GEMM is the shape (1, M, 1, K, N, 1, 1, 1, 0).

@@ -23,6 +23,7 @@ EXPORTS = (
     "bcnn_pack", "bcnn_stem_fused", "bcnn_gemm_b1", "bcnn_gemm_b1_fused", "bcnn_conv2d_b1", "bcnn_conv2d_b1_fused", "bcnn_conv2d_b1_module",
     "bcnn_conv2d_b1_branches", "bcnn_dwconv3x3_module", "bcnn_avgpool", "bcnn_gap", "bcnn_fc",
     "bcnn_prepared_weights_bytes", "bcnn_prepare_weights", "bcnn_conv2d_b1_prepared", "bcnn_gemm_b1_prepared", "bcnn_prepared_preferred",
+    "bcnn_conv2d_b1_fused_noalloc",
     "bcnn_conv2d_b1_engine", "bcnn_gemm_b1_engine", "bcnn_auto_engine", "bcnn_device_error", "bcnn_device_status",
     "bcnn_workspace_bytes", "bcnn_selftest_wait_timeout", "bcnn_status_string", "bcnn_version",
 )
@@ -66,6 +67,7 @@ def load() -> ctypes.CDLL:
         lib.bcnn_conv2d_b1_prepared.argtypes = [vp, vp, vp, vp] + [i32] * 9 + [vp]
         lib.bcnn_gemm_b1_prepared.argtypes = [vp, vp, vp, vp, i64, i32, i32, vp]
         lib.bcnn_prepared_preferred.argtypes = [i32] * 10
+        lib.bcnn_conv2d_b1_fused_noalloc.argtypes = [vp, vp, vp, vp] + [i32] * 9 + [vp]
         lib.bcnn_conv2d_b1_engine.argtypes = [i32, vp, vp, vp, vp] + [i32] * 9 + [vp]
         lib.bcnn_gemm_b1_engine.argtypes = [i32, vp, vp, vp, vp, i64, i32, i32, vp]
         lib.bcnn_auto_engine.argtypes = [i32] * 10
@@ -211,6 +213,19 @@ def bcnn_conv2d_b1_prepared(x_bits, prepared, thr, out, B, H, W, C_in, C_out, kh
 def bcnn_gemm_b1_prepared(A_bits, prepared, thr, out, M, N, K):
     _check(load().bcnn_gemm_b1_prepared(_p(A_bits), _p(prepared), _p(thr), _p(out), M, N, K, _stream()), "bcnn_gemm_b1_prepared")
     return out
+
+
+STATIC_SCRATCH_BYTES = 4 << 20
+
+
+def bcnn_conv2d_b1_fused_noalloc(x_bits, w_bits, thr, y_bits, B, H, W, C_in, C_out, kh, kw, stride, pad):
+    """``bcnn_conv2d_b1_fused`` for callers that cannot allocate: the prepared weights live in a static array of the
+    library (4 MiB per GPU); layers whose prepared form is larger raise BCNN_ERR_WORKSPACE."""
+    if thr is None:
+        raise BcnnError(-1, "bcnn_conv2d_b1_fused_noalloc")
+    _check(load().bcnn_conv2d_b1_fused_noalloc(_p(x_bits), _p(w_bits), _p(thr), _p(y_bits), B, H, W, C_in, C_out, kh, kw,
+                                               stride, pad, _stream()), "bcnn_conv2d_b1_fused_noalloc")
+    return y_bits
 
 
 def bcnn_prepared_preferred(B, H, W, C_in, C_out, kh, kw, stride, pad, fused=True) -> bool:

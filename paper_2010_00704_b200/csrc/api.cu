@@ -349,6 +349,19 @@ int bcnn_gemm_b1_prepared(const void *A_bits, const void *prepared, const int32_
     return launch_conv_tc_pre(p, prepared, static_cast<cudaStream_t>(stream));
 }
 
+int bcnn_conv2d_b1_fused_noalloc(const void *x_bits, const void *w_bits, const int32_t *thr, void *y_bits,
+                                 int B, int H, int W, int C_in, int C_out, int kh, int kw, int stride, int pad,
+                                 void *stream)
+{
+    if (!thr) return BCNN_ERR_INVALID_ARG;
+    ConvProblem p;
+    const int st = make_conv_problem(p, x_bits, w_bits, thr, y_bits, B, H, W, C_in, C_out, kh, kw, stride, pad, true);
+    if (st != BCNN_OK) return st;
+    static_assert(BCNN_STATIC_SCRATCH_BYTES == (4u << 20), "header and kernel file agree on the array's size");
+    if (static_prepared_capacity() != BCNN_STATIC_SCRATCH_BYTES) return BCNN_ERR_CUDA;
+    return launch_conv_tc_pre_static(p, static_cast<cudaStream_t>(stream));
+}
+
 int bcnn_prepared_preferred(int B, int H, int W, int C_in, int C_out, int kh, int kw, int stride, int pad, int fused)
 {
     ConvProblem p;
@@ -413,7 +426,7 @@ const char *bcnn_status_string(int status)
     case BCNN_ERR_UNSUPPORTED: return "unsupported shape or engine";
     case BCNN_ERR_ALIGNMENT: return "pointer not 16-byte aligned";
     case BCNN_ERR_CUDA: return "CUDA runtime error";
-    case BCNN_ERR_WORKSPACE: return "workspace too small";
+    case BCNN_ERR_WORKSPACE: return "workspace too small (the layer's prepared weights exceed the library's static scratch array)";
     case BCNN_ERR_TIMEOUT: return "a bounded device-side wait gave up";
     // device error word: which bounded wait gave up
     case 101: return "device wait timed out: streaming tcgen05 engine, producer waiting for a free ring slot";

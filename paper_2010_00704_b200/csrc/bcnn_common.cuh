@@ -106,6 +106,8 @@ void prepared_layout(int C_out, int K, PreparedWeights &pw, size_t &bytes);
 int launch_prepare_weights(const uint32_t *w, void *prepared, int C_out, int K, cudaStream_t stream);
 int launch_conv_tc_pre(const ConvProblem &p, const void *prepared, cudaStream_t stream);
 bool conv_tc_pre_supports(const ConvProblem &p);
+int launch_conv_tc_pre_static(const ConvProblem &p, cudaStream_t stream);   // prepared weights in the library's static array
+size_t static_prepared_capacity();
 bool conv_tc_i8_supports(const ConvProblem &p);
 int launch_selftest_wait_timeout(int polls, cudaStream_t stream);
 int launch_conv_branches(const BranchProblem &p, cudaStream_t stream);

@@ -493,6 +493,49 @@ int launch_prepare_weights(const uint32_t *w, void *prepared, int C_out, int K, 
     return cudaGetLastError() == cudaSuccess ? BCNN_OK : BCNN_ERR_CUDA;
 }
 
+// ---- the variant that allocates nothing -------------------------------------------------------------------------
+// Some callers cannot hand the library a buffer for the prepared weights because they cannot allocate device memory
+// at all at the point where they call: code that runs inside somebody else's memory plan (an inference server whose
+// arena is sized before the model's layers are known, a plug-in that only ever receives its input and output
+// tensors), or code running while allocation is forbidden or would synchronise the device.  For them the prepared
+// form lives in this array: it is part of the library's image, so every GPU that loads the library holds these
+// STATIC_PREPARED_BYTES until the process exits.  The host-side name of a __device__ array is only a stand-in; the
+// kernels need its device address, fetched once per device with cudaGetSymbolAddress.
+constexpr size_t STATIC_PREPARED_BYTES = (size_t)4 << 20;
+static __device__ __align__(256) unsigned char g_static_prepared[STATIC_PREPARED_BYTES];
+
+size_t static_prepared_capacity() { return STATIC_PREPARED_BYTES; }
+
+// Device address of the array on the current device (nullptr on failure); looked up on a device's first call.
+static void *static_prepared_address()
+{
+    static void *cache[64] = {nullptr};
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+    if (!cache[dev]) {
+        void *ptr = nullptr;
+        if (cudaGetSymbolAddress(&ptr, g_static_prepared) != cudaSuccess) return nullptr;
+        cache[dev] = ptr;
+    }
+    return cache[dev];
+}
+
+int launch_conv_tc_pre_static(const ConvProblem &p, cudaStream_t stream)
+{
+    if (!conv_tc_pre_supports(p)) return BCNN_ERR_UNSUPPORTED;
+    PreparedWeights pw;
+    size_t bytes = 0;
+    prepared_layout(p.C_out, p.K, pw, bytes);
+    if (bytes > STATIC_PREPARED_BYTES) return BCNN_ERR_WORKSPACE;
+    void *scratch = static_prepared_address();
+    if (!scratch) return BCNN_ERR_CUDA;
+    // the expansion rewrites every byte of the layout it uses (padding rows and K words as zeros), so nothing of an
+    // earlier call's contents is ever read
+    const int st = launch_prepare_weights(p.w, scratch, p.C_out, p.K, stream);
+    if (st != BCNN_OK) return st;
+    return launch_conv_tc_pre(p, scratch, stream);
+}
+
 bool conv_tc_pre_supports(const ConvProblem &p)
 {
     if (p.mode != 0 && p.mode != 1) return false;
