@@ -80,6 +80,29 @@ class FusedChain:
         else:
             binding.bcnn_pack(x_real, self.bias, self.in_bits, self.batch, H, W, C, self.replicate)
 
+    def enqueue_layer(self, i: int, cur):
+        """Enqueue layer i (input ``cur``, output ``self.outs[i]``): the prepared call where its weights were prepared,
+        else the plain fused call."""
+        l, o = self.layers[i], self.outs[i]
+        if self.prepared[i] is not None:
+            binding.bcnn_conv2d_b1_prepared(cur, self.prepared[i], self.thr[i], o, self.batch, l.H, l.W, l.C_in, l.C_out,
+                                            l.k, l.k, l.stride, l.pad)
+        else:
+            binding.bcnn_conv2d_b1_fused(cur, self.w[i], self.thr[i], o, self.batch, l.H, l.W, l.C_in, l.C_out, l.k, l.k,
+                                         l.stride, l.pad, engine=self.engine)
+        return o
+
+    def engine_name(self, i: int) -> str:
+        """Name of the engine layer i runs on."""
+        l = self.layers[i]
+        if i == 0 and self.fuse_stem:
+            return "stem"
+        if self.prepared[i] is not None:
+            return "tc_pre"
+        if self.engine != binding.ENGINE_AUTO:
+            return {v: k for k, v in binding.ENGINES.items()}[self.engine]
+        return binding.bcnn_auto_engine(self.batch, l.H, l.W, l.C_in, l.C_out, l.k, l.k, l.stride, l.pad)
+
     def enqueue(self, include_pack: bool = True):
         """Enqueue the whole sequence on the current stream; returns the last layer's packed output."""
         if self.x_real is not None and include_pack:
@@ -89,13 +112,7 @@ class FusedChain:
             if i == 0 and self.fuse_stem:        # done by enqueue_pack
                 cur = o
                 continue
-            if self.prepared[i] is not None:
-                binding.bcnn_conv2d_b1_prepared(cur, self.prepared[i], t, o, self.batch, l.H, l.W, l.C_in, l.C_out, l.k, l.k,
-                                                l.stride, l.pad)
-            else:
-                binding.bcnn_conv2d_b1_fused(cur, w, t, o, self.batch, l.H, l.W, l.C_in, l.C_out, l.k, l.k,
-                                             l.stride, l.pad, engine=self.engine)
-            cur = o
+            cur = self.enqueue_layer(i, cur)
         return cur
 
     def capture(self):
