@@ -112,6 +112,8 @@ int dispatch(int engine, const ConvProblem &p, cudaStream_t stream)
         return launch_conv_tc_ws(p, stream);
     case BCNN_ENGINE_TC_PW:
         return launch_conv_tc_pw(p, stream);
+    case BCNN_ENGINE_TC_C3:
+        return launch_conv_tc_c3(p, stream);
     default:
         return BCNN_ERR_UNSUPPORTED;
     }
@@ -445,6 +447,12 @@ const char *bcnn_status_string(int status)
     case 134: return "device wait timed out: prepared-weights tcgen05 engine, loader waiting for a free ring slot";
     case 125: return "device wait timed out: pointwise tcgen05 engine, producer waiting for a slot's previous MMAs";
     case 126: return "device wait timed out: pointwise tcgen05 engine, issuer waiting for a slot's accumulators";
+    case 141: return "device wait timed out: 3x3 halo-tile tcgen05 engine, loader waiting for a free ring stage";
+    case 142: return "device wait timed out: 3x3 halo-tile tcgen05 engine, producer waiting for a tile's halo";
+    case 143: return "device wait timed out: 3x3 halo-tile tcgen05 engine, issuer waiting for a slot's expanded rows";
+    case 144: return "device wait timed out: 3x3 halo-tile tcgen05 engine, epilogue waiting for a chunk's accumulators";
+    case 145: return "device wait timed out: 3x3 halo-tile tcgen05 engine, producer waiting for a slot's previous MMAs";
+    case 146: return "device wait timed out: 3x3 halo-tile tcgen05 engine, issuer waiting for a slot's accumulators";
     case BCNN_SELFTEST_TIMEOUT_CODE: return "device wait timed out: self-test (expected)";
     default: return status > 0 ? "device-side error code" : "unknown status";
     }
