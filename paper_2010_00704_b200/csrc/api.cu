@@ -76,6 +76,8 @@ int make_conv_problem(ConvProblem &p, const void *x, const void *w, const int32_
 // Measured on B200 (bench.py --mode sweep):
 //   * pointwise layers (1x1, stride 1, no padding; GEMMs) with K <= 128 and C_out <= 128, packed output: pointwise
 //     tcgen05 engine (memory-bound shapes: rows bulk-copied in chunks, one hand-over per chunk);
+//   * 3x3 layers (stride 1 or 2) on 32 or 64 input channels with C_out <= 64, packed output, whose 8 x 16 output tiles
+//     are at least three quarters full: halo-tile tcgen05 engine (input tiles by tiled TMA copies);
 //   * C_out >= 256, or weights too large to keep expanded in shared memory: streaming tcgen05 engine;
 //   * 1x1 layer with C_in = 32 and C_out <= 32 (one XOR + popcount per output): CUDA-core pointwise kernel;
 //   * C_out <= 128 with K >= 64, and wider layers with K <= 1152 and M >= 32768 (in 128-channel slices):
@@ -85,6 +87,10 @@ int make_conv_problem(ConvProblem &p, const void *x, const void *w, const int32_
 int auto_engine(const ConvProblem &p)
 {
     if (conv_tc_pw_supports(p)) return BCNN_ENGINE_TC_PW;
+    if (p.C_out <= 64 && conv_tc_c3_supports(p)) {
+        const long covered = (long)((p.OH + 7) / 8 * 8) * ((p.OW + 15) / 16 * 16);
+        if (4L * p.OH * p.OW >= 3L * covered) return BCNN_ENGINE_TC_C3;
+    }
     if (conv_lop3_pointwise_k32(p)) return BCNN_ENGINE_LOP3;
     if (p.C_out <= 128 && p.K >= 64 && conv_tc_ws_supports(p)) return BCNN_ENGINE_TC_WS;
     // wider layers in slices of 128 output channels: ahead of the streaming engine while K is short and there are
@@ -449,10 +455,10 @@ const char *bcnn_status_string(int status)
     case 126: return "device wait timed out: pointwise tcgen05 engine, issuer waiting for a slot's accumulators";
     case 141: return "device wait timed out: 3x3 halo-tile tcgen05 engine, loader waiting for a free ring stage";
     case 142: return "device wait timed out: 3x3 halo-tile tcgen05 engine, producer waiting for a tile's halo";
-    case 143: return "device wait timed out: 3x3 halo-tile tcgen05 engine, issuer waiting for a slot's expanded rows";
-    case 144: return "device wait timed out: 3x3 halo-tile tcgen05 engine, epilogue waiting for a chunk's accumulators";
-    case 145: return "device wait timed out: 3x3 halo-tile tcgen05 engine, producer waiting for a slot's previous MMAs";
-    case 146: return "device wait timed out: 3x3 halo-tile tcgen05 engine, issuer waiting for a slot's accumulators";
+    case 143: return "device wait timed out: 3x3 halo-tile tcgen05 engine, issuer waiting for a tile's expanded rows";
+    case 144: return "device wait timed out: 3x3 halo-tile tcgen05 engine, epilogue waiting for a tile's accumulator";
+    case 145: return "device wait timed out: 3x3 halo-tile tcgen05 engine, producer waiting for an activation stage's previous MMAs";
+    case 146: return "device wait timed out: 3x3 halo-tile tcgen05 engine, issuer waiting for an accumulator";
     case BCNN_SELFTEST_TIMEOUT_CODE: return "device wait timed out: self-test (expected)";
     default: return status > 0 ? "device-side error code" : "unknown status";
     }

@@ -14,20 +14,30 @@
 // Arithmetic as in the pointwise engine (conv_tc_pw.cu): unsigned activation bytes {0, 2^j} against signed weight bytes,
 // every product +-64, the per-channel constant written by a first MMA against a constant activation tile.
 //
-// The CTA runs TWO independent pipelines (slots); tiles alternate between them.  A slot owns a loader warp with a ring
-// of halo tiles, four producer warps, an issuer warp, four epilogue warps and its share of tensor memory: NACC
-// accumulators and a ring of NU activation UNITS of UW words of K (8 columns per word).  A tile's K is cut into
-// UPT = ceil(9 C_in / 32 / UW) units.  The producers fill units in order, the issuer multiplies a unit as soon as it is
-// full and hands it back with a commit, the last unit's commit also hands the accumulator to the epilogue; so inside a
-// slot the expansion of the next unit (or tile) runs under the MMAs of this one, and the epilogue of a tile under the
-// MMAs of the next (NACC = 2).  An issuer that waits right behind its own MMAs stalls until they drain; the other
-// slot's MMAs fill that gap.
+// One MMA stream, one commit per tile.  Tensor memory holds NACC accumulators and a ring of NA activation tiles (72
+// columns per 32 input channels).  One issuer warp walks the CTA's tiles in order: it waits until the tile's activations
+// are full and its accumulator free, issues the tile's MMAs and ONE commit on the tile's "done" barrier, which both the
+// epilogue (accumulator ready) and the producers (activation stage free again) wait on: a tcgen05.commit costs the
+// issuing thread about a hundred cycles, and a wait on a barrier that is already complete almost nothing, so with the
+// producers ahead the MMAs of consecutive tiles queue back to back.  Two loader warps and two epilogue groups take
+// alternate tiles.  C_in = 64: both producer groups (four warps each) work on EVERY tile - group 0 expands taps 0..4,
+// group 1 taps 5..8 of the same 128 pixels - which halves the time a tile takes to fill; with only two or three
+// activation tiles in tensor memory that time matters.  C_in = 32: the producer groups take alternate tiles (fewer
+// instructions per tile), and so do two issuer warps: there a tile's MMAs take 160 - 320 cycles and one issuer's
+// waits and commit would be the bound.
+// The "done" barriers form a ring of NB = 8 (tile n -> barrier n % 8): a multiple of NACC and at least NA, so that
+// neither waiter can be lapped.
 // K = 288 or 576 makes |accumulator| exceed 16 bits, so the epilogue reads 32-bit accumulators and shifts sign bits in.
 // A parity wait on an mbarrier is only right while the waiter starts waiting for completion k after completion k - 1 and
-// before completion k + 1: every barrier here has one group of waiters that takes its completions in turn.
+// before completion k + 1.  Tile n's "done" is completion n / 8 of its barrier; its waiters are the epilogue of tile n
+// and the producers of tile n + NA.  Both have seen tile n - 2 done (an issuer's tiles complete in order: so is tile
+// n - 8), and tile n + 8 cannot be issued before both are through: its issuer first issues tile n + NA (the same
+// issuer: NA is a multiple of the number of issuers), which needs that tile's activations, and, NB being a multiple
+// of NACC, tile n + 8 needs the accumulator of tile n back from the epilogue.
 // Every mbarrier wait is bounded and reports through the device error word.
 #include "tc_slot.cuh"
 #include <cuda.h>
+#include <type_traits>
 
 namespace bcnn {
 
@@ -37,36 +47,46 @@ using namespace tc;
 
 constexpr int ERR_C3_LOADER_TIMEOUT = 141;       // loader: no free ring stage
 constexpr int ERR_C3_PRODUCER_TIMEOUT = 142;     // producer: the tile's halo did not arrive
-constexpr int ERR_C3_ISSUER_TIMEOUT = 143;       // issuer: a unit was not filled
+constexpr int ERR_C3_ISSUER_TIMEOUT = 143;       // issuer: a tile's activations were not filled
 constexpr int ERR_C3_EPILOGUE_TIMEOUT = 144;     // epilogue: the tile's MMAs did not complete
-constexpr int ERR_C3_UNIT_TIMEOUT = 145;         // producer: a unit's previous MMAs did not complete
+constexpr int ERR_C3_UNIT_TIMEOUT = 145;         // producer: the activation stage's previous MMAs did not complete
 constexpr int ERR_C3_ACC_TIMEOUT = 146;          // issuer: an accumulator was not handed back
 
 constexpr int TH = 8, TW = 16;            // output tile (TH * TW = 128 = tensor-memory lanes)
-constexpr int NSLOT = 2;
-constexpr int RD = 6;                     // halo tiles in a slot's ring
+constexpr int NGRP = 2;                   // loader / epilogue groups (alternate tiles); producer groups (taps 0..4 / 5..8 of every tile)
+constexpr int TAP_SPLIT = 5;
+constexpr int RD = 6;                     // halo tiles in a group's ring
 constexpr int CONST_COLS = 8;
-constexpr int MAX_NU = 3, MAX_NACC = 2;
+constexpr int NB = 8;                     // ring of "tile done" barriers
+constexpr int MAX_NA = 5, MAX_NACC = 4;
 
-// CW: words per input pixel (1, 2); BN: accumulator columns per tile (32, 64, 128 >= C_out).
+// CW: words per input pixel (1, 2) = units per tile; BN: accumulator columns per tile (32, 64, 128 >= C_out).
 template <int CW, int BN> struct C3Cfg {
     static constexpr int KW = 9 * CW;                       // words of K per row
     static constexpr int KT = (KW + 3) / 4;                 // 128-byte stages of the expanded weights
-    static constexpr int NACC = BN == 128 ? 1 : 2;          // accumulators per slot
-    static constexpr int UW = BN == 32 ? 9 : 5;             // words per unit
-    static constexpr int NU = BN == 32 ? 2 : 3;             // units in a slot's ring
-    static constexpr int UPT = (KW + UW - 1) / UW;          // units per tile
-    static constexpr int U_COLS = 8 * UW;
-    static constexpr int SLOT_COLS = NACC * BN + NU * U_COLS;
-    static constexpr int C_COL = NSLOT * SLOT_COLS;         // the constant activation tile
+    static constexpr int A_COLS = 8 * KW;                   // columns of one activation tile
+    static constexpr int NACC = CW == 2 && BN == 128 ? 1 : (CW == 1 && BN == 32 ? 4 : 2);   // accumulators
+    static constexpr int NA0 = (512 - CONST_COLS - NACC * BN) / A_COLS;
+    // C_in = 64 (MMA-bound tiles): one issuer; both producer groups fill every tile (COOP).  C_in = 32 (short tiles, bound
+    // by instruction issue): two issuer warps and the producer groups take alternate tiles; then a tile and the next user
+    // of its activation stage must belong to the same issuer, so the ring has an even number of stages.
+    static constexpr bool COOP = CW == 2;
+    // K = 288: |accumulator| <= 32 (2 K + 1) < 2^15, so the epilogue can read packed 16-bit halves and gather sign bits
+    // with byte permutes (half the logic operations); the weight rows are then laid out in the gathering's column order
+    static constexpr bool PACK16 = CW == 1;
+    static constexpr int NISS = CW == 2 ? 1 : 2;
+    static constexpr int NA1 = NA0 > MAX_NA ? MAX_NA : NA0;
+    static constexpr int NA = NISS == 2 ? NA1 / 2 * 2 : NA1;   // activation tiles in the ring: 4, 4, 2 (C_in 32); 3, 2, 2 (C_in 64)
+    static constexpr int A_COL0 = NACC * BN;
+    static constexpr int C_COL = A_COL0 + NA * A_COLS;      // the constant activation tile
     static_assert(C_COL + CONST_COLS <= 512, "tensor memory budget");
-    static_assert(NU <= MAX_NU && NACC <= MAX_NACC, "barrier table");
-    // warps: 0, 1 issuers; 2, 3 loaders; then per slot four producer warps, then per slot four epilogue warps
-    // (groups start at multiples of four: warp % 4 is the tensor-memory lane quadrant of a warp)
+    static_assert(NA >= 2 && NA <= NB && NB % NACC == 0 && NACC <= MAX_NACC && NACC % NISS == 0 && NA % NISS == 0, "barrier rings");
+    // warps: 0 (and 1) issuers, 2 and 3 loaders, then per group four producer warps, then per group four epilogue
+    // warps (groups start at multiples of four: warp % 4 is the tensor-memory lane quadrant of a warp)
     static constexpr int FIRST_LOADER_WARP = 2;
     static constexpr int FIRST_PRODUCER_WARP = 4;
-    static constexpr int FIRST_EPILOGUE_WARP = 4 + 4 * NSLOT;
-    static constexpr int WARPS = 4 + 8 * NSLOT;
+    static constexpr int FIRST_EPILOGUE_WARP = 4 + 4 * NGRP;
+    static constexpr int WARPS = 4 + 8 * NGRP;
     static constexpr int THREADS = 32 * WARPS;
     static constexpr int W_TILE_BYTES = BN * ROWB;
 };
@@ -99,26 +119,7 @@ template <int CW, int BN>
 int c3_smem_bytes(const C3Geom &g)
 {
     using C = C3Cfg<CW, BN>;
-    return 1024 + (C::KT + 1) * C::W_TILE_BYTES + NSLOT * RD * g.stage_bytes + 128;
-}
-
-// tensor-memory stores of n expanded words (8 columns each) starting at taddr, no wait
-template <int N>
-__device__ __forceinline__ void store_words(uint32_t taddr, const uint32_t *wds)
-{
-#pragma unroll
-    for (int e4 = 0; e4 + 4 <= N; e4 += 4) {
-        uint32_t v[32];
-#pragma unroll
-        for (int e = 0; e < 4; ++e) expand_a(wds[e4 + e], &v[8 * e]);
-        tc_st32_nowait(taddr + 8u * e4, v);
-    }
-#pragma unroll
-    for (int e = N / 4 * 4; e < N; ++e) {
-        uint32_t v[8];
-        expand_a(wds[e], v);
-        tc_st8_nowait(taddr + 8u * e, v);
-    }
+    return 1024 + (C::KT + 1) * C::W_TILE_BYTES + NGRP * RD * g.stage_bytes + 128;
 }
 
 template <int CW, int BN>
@@ -126,47 +127,40 @@ __global__ void __launch_bounds__(C3Cfg<CW, BN>::THREADS, 1)
 conv_tc_c3_kernel(const ConvProblem p, const C3Geom g, const __grid_constant__ CUtensorMap xmap)
 {
     using C = C3Cfg<CW, BN>;
-    constexpr int KW = C::KW, KT = C::KT, NACC = C::NACC, UW = C::UW, NU = C::NU, UPT = C::UPT;
-    constexpr int BARS_PER_SLOT = 2 * RD + 2 * MAX_NU + 2 * MAX_NACC;
+    constexpr int KW = C::KW, KT = C::KT, NACC = C::NACC, NA = C::NA;
+    constexpr int NBARS = 2 * NGRP * RD + MAX_NA + NB + MAX_NACC;
 
     extern __shared__ unsigned char smem_raw[];
-    __shared__ __align__(8) unsigned long long bars[NSLOT * BARS_PER_SLOT];
+    __shared__ __align__(8) unsigned long long bars[NBARS];
     __shared__ uint32_t tmem_base_smem;
     __shared__ int abort_flag_smem;
 
     const int tid = threadIdx.x;
     const int warp = tid >> 5, lane = tid & 31;
-    // this CTA's tiles: blockIdx.x + q * gridDim.x; tile q belongs to slot q % 2, the slot's n-th tile is q = 2 n + slot
+    // this CTA's tiles: blockIdx.x + n * gridDim.x, n = 0, 1, ...; tile n belongs to loader / epilogue group n % 2, uses
+    // accumulator n % NACC, activation stage n % NA and "done" barrier n % NB
     const int my_tiles = (int)blockIdx.x < g.total_tiles ? (g.total_tiles - 1 - (int)blockIdx.x) / (int)gridDim.x + 1 : 0;
     const int cn = min(BN, p.C_out);
 
     const uint32_t wexp = (smem_u32(smem_raw) + 1023u) & ~1023u;          // [KT][BN rows][128 B] expanded weights
     const uint32_t cexp = wexp + KT * C::W_TILE_BYTES;                    // [BN rows][128 B] constant bytes (first 32 of a row)
-    const uint32_t ring = cexp + C::W_TILE_BYTES;                         // [NSLOT][RD] halo tiles
+    const uint32_t ring = cexp + C::W_TILE_BYTES;                         // [NGRP][RD] halo tiles
     const uint32_t bar0 = smem_u32(bars);
-    auto load_full = [&](int sl, int s) { return bar0 + 8u * (sl * BARS_PER_SLOT + s); };
-    auto load_empty = [&](int sl, int s) { return bar0 + 8u * (sl * BARS_PER_SLOT + RD + s); };
-    auto a_full = [&](int sl, int s) { return bar0 + 8u * (sl * BARS_PER_SLOT + 2 * RD + s); };
-    auto a_empty = [&](int sl, int s) { return bar0 + 8u * (sl * BARS_PER_SLOT + 2 * RD + MAX_NU + s); };
-    auto acc_full = [&](int sl, int s) { return bar0 + 8u * (sl * BARS_PER_SLOT + 2 * RD + 2 * MAX_NU + s); };
-    auto acc_free = [&](int sl, int s) { return bar0 + 8u * (sl * BARS_PER_SLOT + 2 * RD + 2 * MAX_NU + MAX_NACC + s); };
+    auto load_full = [&](int gr, int s) { return bar0 + 8u * (gr * RD + s); };
+    auto load_empty = [&](int gr, int s) { return bar0 + 8u * (NGRP * RD + gr * RD + s); };
+    auto a_full = [&](int s) { return bar0 + 8u * (2 * NGRP * RD + s); };
+    auto tile_done = [&](int s) { return bar0 + 8u * (2 * NGRP * RD + MAX_NA + s); };
+    auto acc_free = [&](int s) { return bar0 + 8u * (2 * NGRP * RD + MAX_NA + NB + s); };
     volatile int *abort_flag = &abort_flag_smem;
 
     if (tid == 0) {
-        for (int sl = 0; sl < NSLOT; ++sl) {
-            for (int s = 0; s < RD; ++s) {
-                mbar_init(load_full(sl, s), 1);         // the loader's arrive (+ the copy's bytes)
-                mbar_init(load_empty(sl, s), 4);        // the slot's four producer warps
-            }
-            for (int s = 0; s < MAX_NU; ++s) {
-                mbar_init(a_full(sl, s), 4);            // the slot's four producer warps
-                mbar_init(a_empty(sl, s), 1);           // the issuer's commit
-            }
-            for (int s = 0; s < MAX_NACC; ++s) {
-                mbar_init(acc_full(sl, s), 1);          // the issuer's commit
-                mbar_init(acc_free(sl, s), 4);          // the slot's four epilogue warps
-            }
+        for (int s = 0; s < NGRP * RD; ++s) {
+            mbar_init(load_full(0, s), 1);              // the loader's arrive (+ the copy's bytes)
+            mbar_init(load_empty(0, s), C::COOP ? 8 : 4);   // the producer warps that read the stage
         }
+        for (int s = 0; s < MAX_NA; ++s) mbar_init(a_full(s), C::COOP ? 8 : 4);   // the producer warps that fill the stage
+        for (int s = 0; s < NB; ++s) mbar_init(tile_done(s), 1);        // the issuer's commit
+        for (int s = 0; s < MAX_NACC; ++s) mbar_init(acc_free(s), 4);   // the four epilogue warps of the tile's group
         abort_flag_smem = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -176,8 +170,9 @@ conv_tc_c3_kernel(const ConvProblem p, const C3Geom g, const __grid_constant__ C
     }
     // ---- one-off: expanded weights (K word e -> stage e / 4, 32-byte piece e % 4) and the constant bytes
     for (int idx = tid; idx < (KT + 1) * BN; idx += C::THREADS) {
-        const int kt = idx / BN, row = idx - kt * BN;
-        const bool have = row < cn;
+        const int kt = idx / BN, row = idx - kt * BN;       // MMA row `row` carries channel ch
+        const int ch = C::PACK16 ? (row & ~31) + channel_of_column(row & 31) : row;
+        const bool have = ch < cn;
         const int xr = row & 7;
         if (kt < KT) {
             const uint32_t row_addr = wexp + (uint32_t)kt * C::W_TILE_BYTES + (uint32_t)row * ROWB;
@@ -185,7 +180,7 @@ conv_tc_c3_kernel(const ConvProblem p, const C3Geom g, const __grid_constant__ C
             for (int e = 0; e < 4; ++e) {
                 const int kword = kt * 4 + e;
                 const bool live = kword < KW && have;
-                const uint32_t w = live ? __ldg(p.w + (long)row * KW + kword) : 0u;
+                const uint32_t w = live ? __ldg(p.w + (long)ch * KW + kword) : 0u;
                 expand_store_w_signed(w, live, row_addr, xr, 2 * e);
             }
         } else {
@@ -193,8 +188,8 @@ conv_tc_c3_kernel(const ConvProblem p, const C3Geom g, const __grid_constant__ C
             // all 32, so the row's 32 signed bytes add up to c: c / 32 everywhere, one more unit of c's sign in |c % 32|
             int pop = 0;
             if (have)
-                for (int e = 0; e < KW; ++e) pop += __popc(__ldg(p.w + (long)row * KW + e));
-            int t = have ? __ldg(p.thr + row) : 0;
+                for (int e = 0; e < KW; ++e) pop += __popc(__ldg(p.w + (long)ch * KW + e));
+            int t = have ? __ldg(p.thr + ch) : 0;
             t = max(min(t, p.K + 1), -p.K - 1);
             const int c = have ? p.K - 2 * pop - t : 0;
             const int base = c / 32, rem = c - 32 * base, unit = rem < 0 ? -1 : 1, nrem = rem < 0 ? -rem : rem;
@@ -235,90 +230,103 @@ conv_tc_c3_kernel(const ConvProblem p, const C3Geom g, const __grid_constant__ C
         oh0 = (int)ty * TH;
         ow0 = (int)(rem - ty * (unsigned)g.tiles_x) * TW;
     };
-    auto slot_tiles = [&](int slot) { return (my_tiles + 1 - slot) / 2; };
-    auto tile_of = [&](int slot, int n) { return (int)blockIdx.x + (2 * n + slot) * (int)gridDim.x; };
+    auto tile_of = [&](int n) { return (int)blockIdx.x + n * (int)gridDim.x; };
 
-    if (warp < NSLOT) {
-        // ------------------------------------------------------------------ MMA issuer of slot `warp`
-        const int slot = warp;
+    if (warp < C::NISS) {
+        // ------------------------------------------------------------------ MMA issuer of tiles n = warp (mod NISS), in order
         constexpr uint32_t idesc = make_idesc(BN) | (1u << 10);                  // B operand: signed bytes
         const uint64_t desc0 = make_desc(wexp);
         const uint32_t desc_hi = (uint32_t)(desc0 >> 32), b_lo = (uint32_t)desc0;
         const uint32_t c_lo = (uint32_t)make_desc(cexp);
-        const uint32_t tmem_u = __shfl_sync(0xffffffffu, tmem_base, 0) + (uint32_t)(slot * C::SLOT_COLS);
-        const uint32_t c_t = tmem_u - (uint32_t)(slot * C::SLOT_COLS) + (uint32_t)C::C_COL;
-        const int nt = slot_tiles(slot);
-        int ust = 0, acc = 0;
-        uint32_t uphase = 0, aphase = 0;          // parity of the unit ring's / the accumulators' current round
-        bool ok = true;
-        for (int n = 0; n < nt && ok; ++n) {
-            const uint32_t d_t = tmem_u + (uint32_t)(acc * BN);
+        const uint32_t tmem_u = __shfl_sync(0xffffffffu, tmem_base, 0);
+        const uint32_t c_t = tmem_u + (uint32_t)C::C_COL;
+        for (int n = warp; n < my_tiles; n += C::NISS) {
+            const int ast = n % NA, acc = n % NACC;
+            if (!pw_wait(a_full(ast), (uint32_t)(n / NA) & 1u, abort_flag, p.err, ERR_C3_ISSUER_TIMEOUT)) break;
+            // the epilogue has read the accumulator's previous tile
+            if (n >= NACC && !pw_wait(acc_free(acc), (uint32_t)(n / NACC - 1) & 1u, abort_flag, p.err, ERR_C3_ACC_TIMEOUT)) break;
+            tc_fence_after();
+            if (elect_one()) {
+                const uint32_t d_t = tmem_u + (uint32_t)(acc * BN);
+                const uint32_t a_t = tmem_u + (uint32_t)(C::A_COL0 + ast * C::A_COLS);
+                tc_mma_i8_ts(d_t, c_t, c_lo, desc_hi, idesc, 0u);               // accumulator = the per-channel constants
 #pragma unroll
-            for (int h = 0; h < UPT; ++h) {
-                ok = pw_wait(a_full(slot, ust), uphase, abort_flag, p.err, ERR_C3_ISSUER_TIMEOUT);
-                if (!ok) break;
-                if (h == 0 && n >= NACC) {       // the epilogue has read the accumulator's previous tile
-                    ok = pw_wait(acc_free(slot, acc), aphase ^ 1u, abort_flag, p.err, ERR_C3_ACC_TIMEOUT);
-                    if (!ok) break;
-                }
-                tc_fence_after();
-                if (elect_one()) {
-                    const uint32_t a_t = tmem_u + (uint32_t)(NACC * BN + ust * C::U_COLS);
-                    if (h == 0) tc_mma_i8_ts(d_t, c_t, c_lo, desc_hi, idesc, 0u);   // accumulator = the per-channel constants
-#pragma unroll
-                    for (int e = h * UW; e < (h + 1) * UW && e < KW; ++e)
-                        tc_mma_i8_ts(d_t, a_t + 8u * (e - h * UW), b_lo + (uint32_t)((e >> 2) * (C::W_TILE_BYTES >> 4) + 2 * (e & 3)), desc_hi, idesc, 1u);
-                    tc_commit(a_empty(slot, ust));
-                    if (h == UPT - 1) tc_commit(acc_full(slot, acc));
-                }
-                __syncwarp();
-                if (++ust == NU) { ust = 0; uphase ^= 1u; }
-            }
-            if (++acc == NACC) { acc = 0; aphase ^= 1u; }
-        }
-    } else if (warp < C::FIRST_PRODUCER_WARP) {
-        // ------------------------------------------------------------------ loader of slot warp - 2: one halo tile per TMA copy
-        const int slot = warp - C::FIRST_LOADER_WARP;
-        const int nt = slot_tiles(slot);
-        int stage = 0;
-        uint32_t phase = 1;                       // first pass through the ring: the stages are free
-        int issued = 0;
-        for (int n = 0; n < nt; ++n) {
-            if (!pw_wait(load_empty(slot, stage), phase, abort_flag, p.err, ERR_C3_LOADER_TIMEOUT)) break;
-            if (lane == 0) {
-                const uint32_t dst = ring + (uint32_t)(slot * RD + stage) * (uint32_t)g.stage_bytes;
-                int b, oh0, ow0;
-                tile_origin(tile_of(slot, n), b, oh0, ow0);
-                const int x = (ow0 * g.stride - p.pad - g.xoff) * CW;        // words; a multiple of 4 by construction
-                const int y = oh0 * g.stride - p.pad;
-                asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(load_full(slot, stage)), "r"((uint32_t)(g.hb * g.wbw * 4)) : "memory");
-                asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
-                             ::"r"(dst), "l"(reinterpret_cast<uint64_t>(&xmap)), "r"(x), "r"(y), "r"(b), "r"(load_full(slot, stage)) : "memory");
+                for (int e = 0; e < KW; ++e)
+                    tc_mma_i8_ts(d_t, a_t + 8u * e, b_lo + (uint32_t)((e >> 2) * (C::W_TILE_BYTES >> 4) + 2 * (e & 3)), desc_hi, idesc, 1u);
+                tc_commit(tile_done(n % NB));
             }
             __syncwarp();
-            ++issued;
-            if (++stage == RD) { stage = 0; phase ^= 1u; }
         }
-        // after a time-out elsewhere: copies still in flight must land before the CTA's shared memory goes away
-        if (*abort_flag) {
-            const int first = issued > RD ? issued - RD : 0;
-            for (int q = first; q < issued; ++q)
-                pw_wait(load_full(slot, q % RD), (uint32_t)(q / RD) & 1u, abort_flag, nullptr, 0);
+    } else if (warp < C::FIRST_LOADER_WARP) {
+        // (idle)
+    } else if (warp < C::FIRST_PRODUCER_WARP) {
+        // ------------------------------------------------------------------ loader of group warp - 2: one halo tile per TMA copy
+        const int grp = warp - C::FIRST_LOADER_WARP;
+        {
+            int stage = 0;
+            uint32_t phase = 1;                       // first pass through the ring: the stages are free
+            int issued = 0;
+            for (int n = grp; n < my_tiles; n += NGRP) {
+                if (!pw_wait<256>(load_empty(grp, stage), phase, abort_flag, p.err, ERR_C3_LOADER_TIMEOUT)) break;
+                if (lane == 0) {
+                    const uint32_t dst = ring + (uint32_t)(grp * RD + stage) * (uint32_t)g.stage_bytes;
+                    int b, oh0, ow0;
+                    tile_origin(tile_of(n), b, oh0, ow0);
+                    const int x = (ow0 * g.stride - p.pad - g.xoff) * CW;        // words; a multiple of 4 by construction
+                    const int y = oh0 * g.stride - p.pad;
+                    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(load_full(grp, stage)), "r"((uint32_t)(g.hb * g.wbw * 4)) : "memory");
+                    asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+                                 ::"r"(dst), "l"(reinterpret_cast<uint64_t>(&xmap)), "r"(x), "r"(y), "r"(b), "r"(load_full(grp, stage)) : "memory");
+                }
+                __syncwarp();
+                ++issued;
+                if (++stage == RD) { stage = 0; phase ^= 1u; }
+            }
+            // after a time-out elsewhere: copies still in flight must land before the CTA's shared memory goes away
+            if (*abort_flag) {
+                const int first = issued > RD ? issued - RD : 0;
+                for (int q = first; q < issued; ++q)
+                    pw_wait(load_full(grp, q % RD), (uint32_t)(q / RD) & 1u, abort_flag, nullptr, 0);
+            }
         }
     } else if (warp >= C::FIRST_EPILOGUE_WARP) {
-        // ------------------------------------------------------------------ epilogue of slot (warp - first) / 4
+        // ------------------------------------------------------------------ epilogue group (warp - first) / 4
         const int quad = warp & 3;
-        const int slot = (warp - C::FIRST_EPILOGUE_WARP) >> 2;
+        const int grp = (warp - C::FIRST_EPILOGUE_WARP) >> 2;
         const int r = quad * 32 + lane;                           // row of the tile = output pixel (r / TW, r % TW)
-        const uint32_t t_lane = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(slot * C::SLOT_COLS);
+        const uint32_t t_lane = tmem_base + ((uint32_t)(quad * 32) << 16);
         const int owords = p.C_out >> 5;
-        const int nt = slot_tiles(slot);
-        int acc = 0;
-        uint32_t aphase = 0;
-        for (int n = 0; n < nt; ++n) {
-            if (!pw_wait(acc_full(slot, acc), aphase, abort_flag, p.err, ERR_C3_EPILOGUE_TIMEOUT)) break;
+        for (int n = grp; n < my_tiles; n += NGRP) {
+            const int acc = n % NACC;
+            if (!pw_wait<128>(tile_done(n % NB), (uint32_t)(n / NB) & 1u, abort_flag, p.err, ERR_C3_EPILOGUE_TIMEOUT)) break;
             tc_fence_after();
             uint32_t words[BN / 32];
+            if constexpr (C::PACK16) {
+                constexpr int NR = BN == 32 ? 16 : 32;                       // registers per load
+                constexpr int NL = BN == 32 ? 1 : BN / 64;                   // loads
+                uint32_t rr[NL][NR];
+                if constexpr (BN == 32) {
+                    tc_ld32_pack16(t_lane + (uint32_t)(acc * BN), rr[0]);
+                } else {
+#pragma unroll
+                    for (int h = 0; h < NL; ++h) tc_ld64_pack16(t_lane + (uint32_t)(acc * BN + h * 64), rr[h]);
+                }
+                tc_wait_ld();
+#pragma unroll
+                for (int h = 0; h < NL; ++h) pin_regs(rr[h]);
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(acc_free(acc));
+                if constexpr (BN == 32) {
+                    words[0] = sign_word(rr[0]);
+                } else {
+#pragma unroll
+                    for (int h = 0; h < NL; ++h) {
+                        words[2 * h] = sign_word(rr[h]);
+                        words[2 * h + 1] = sign_word(rr[h] + 16);
+                    }
+                }
+            } else {
 #pragma unroll
             for (int ch = 0; ch < BN / 32; ++ch) {
                 words[ch] = 0;
@@ -328,7 +336,7 @@ conv_tc_c3_kernel(const ConvProblem p, const C3Geom g, const __grid_constant__ C
                     if ((ch + 1) * 32 >= cn) {                        // the accumulator's last columns are in registers
                         tc_fence_before();
                         __syncwarp();
-                        if (lane == 0) mbar_arrive(acc_free(slot, acc));
+                        if (lane == 0) mbar_arrive(acc_free(acc));
                     }
                     // bit i = (v[i] >= 0): sign bits shifted in, last column first; two chains of 16
                     uint32_t hi = 0, lo = 0;
@@ -340,8 +348,9 @@ conv_tc_c3_kernel(const ConvProblem p, const C3Geom g, const __grid_constant__ C
                     words[ch] = ~__byte_perm(lo, hi, 0x5410);
                 }
             }
+            }
             int b, oh0, ow0;
-            tile_origin(tile_of(slot, n), b, oh0, ow0);
+            tile_origin(tile_of(n), b, oh0, ow0);
             const int oh = oh0 + (r >> 4), ow = ow0 + (r & 15);
             if (oh < p.OH && ow < p.OW) {
                 uint32_t *dst = static_cast<uint32_t *>(p.out) + (((long)b * p.OH + oh) * p.OW + ow) * owords;
@@ -355,60 +364,75 @@ conv_tc_c3_kernel(const ConvProblem p, const C3Geom g, const __grid_constant__ C
                         if (ch < owords) dst[ch] = words[ch];
                 }
             }
-            if (++acc == NACC) { acc = 0; aphase ^= 1u; }
         }
     } else {
-        // ------------------------------------------------------------------ producers of slot (warp - first) / 4
+        // ------------------------------------------------------------------ producer group (warp - first) / 4
         // thread = output pixel (ty, tx) of the tile = tensor-memory lane; its nine input pixels sit at rows
-        // ty * s + kr, pixels tx * s + XOFF + kt of the halo tile
+        // ty * s + kr, pixels tx * s + XOFF + kt of the halo tile.  K word order: tap-major (tap = 3 kr + kt), the
+        // pixel's words within a tap.  Group 0 takes taps 0..4, group 1 taps 5..8 of every tile.
         const int quad = warp & 3;
-        const int slot = (warp - C::FIRST_PRODUCER_WARP) >> 2;
+        const int grp = (warp - C::FIRST_PRODUCER_WARP) >> 2;
         const int r = quad * 32 + lane;
         const uint32_t my_off = (uint32_t)((((r >> 4) * g.stride) * g.wbw + ((r & 15) * g.stride + g.xoff) * CW) * 4);
         const uint32_t row_pitch = (uint32_t)(g.wbw * 4);
-        const uint32_t t_lane = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)(slot * C::SLOT_COLS + NACC * BN);
+        const uint32_t t_lane = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)C::A_COL0;
         const uint32_t lane0 = lane == 0 ? 1u : 0u;
-        const int nt = slot_tiles(slot);
-        int stage = 0, ust = 0, units = 0;
-        uint32_t lphase = 0, uphase = 0;
-        bool ok = true;
-        for (int n = 0; n < nt && ok; ++n) {
-            uint32_t wds[KW];
-            if (!pw_wait(load_full(slot, stage), lphase, abort_flag, p.err, ERR_C3_PRODUCER_TIMEOUT)) break;
-            const uint32_t src = ring + (uint32_t)(slot * RD + stage) * (uint32_t)g.stage_bytes + my_off;
+        // taps [T0, T1) of every tile: W = (T1 - T0) * CW words, tensor-memory columns from 8 * T0 * CW of the stage
+        auto produce = [&](auto t0c, auto t1c, const int n0, const int step) {
+            constexpr int T0 = decltype(t0c)::value, T1 = decltype(t1c)::value, W = (T1 - T0) * CW;
+            for (int n = n0; n < my_tiles; n += step) {
+                const int lg = n & 1, stage = (n >> 1) % RD;
+                uint32_t wds[W];
+                if (!pw_wait<64>(load_full(lg, stage), (uint32_t)((n >> 1) / RD) & 1u, abort_flag, p.err, ERR_C3_PRODUCER_TIMEOUT)) break;
+                const uint32_t src = ring + (uint32_t)(lg * RD + stage) * (uint32_t)g.stage_bytes + my_off;
 #pragma unroll
-            for (int kr = 0; kr < 3; ++kr)
-#pragma unroll
-                for (int kt = 0; kt < 3; ++kt) {
-                    const uint32_t a = src + (uint32_t)kr * row_pitch + (uint32_t)(kt * CW * 4);
+                for (int tap = T0; tap < T1; ++tap) {
+                    const uint32_t a = src + (uint32_t)(tap / 3) * row_pitch + (uint32_t)((tap % 3) * CW * 4);
                     if constexpr (CW == 2) {
-                        asm volatile("ld.shared.v2.b32 {%0,%1}, [%2];" : "=r"(wds[(kr * 3 + kt) * 2]), "=r"(wds[(kr * 3 + kt) * 2 + 1]) : "r"(a) : "memory");
+                        asm volatile("ld.shared.v2.b32 {%0,%1}, [%2];" : "=r"(wds[(tap - T0) * 2]), "=r"(wds[(tap - T0) * 2 + 1]) : "r"(a) : "memory");
                     } else {
-                        asm volatile("ld.shared.b32 %0, [%1];" : "=r"(wds[kr * 3 + kt]) : "r"(a) : "memory");
+                        asm volatile("ld.shared.b32 %0, [%1];" : "=r"(wds[tap - T0]) : "r"(a) : "memory");
                     }
                 }
-            __syncwarp();
-            mbar_arrive_pred(load_empty(slot, stage), lane0);       // the stage may be refilled
-            if (++stage == RD) { stage = 0; lphase ^= 1u; }
+                __syncwarp();
+                mbar_arrive_pred(load_empty(lg, stage), lane0);        // the stage may be refilled
+                // the first four words are expanded before the wait for the activation stage
+                uint32_t v[32];
 #pragma unroll
-            for (int h = 0; h < UPT; ++h) {
-                // the MMAs of the unit's previous use have read it (nothing to wait for the first time round the ring)
-                if (units >= NU) {
-                    ok = pw_wait(a_empty(slot, ust), uphase ^ 1u, abort_flag, p.err, ERR_C3_UNIT_TIMEOUT);
-                    if (!ok) break;
+                for (int e = 0; e < 4; ++e) expand_a(wds[e], &v[8 * e]);
+                // the MMAs of tile n - NA have read the stage (nothing to wait for the first time round the ring)
+                if (n >= NA) {
+                    const int m = n - NA;
+                    if (!pw_wait<64>(tile_done(m % NB), (uint32_t)(m / NB) & 1u, abort_flag, p.err, ERR_C3_UNIT_TIMEOUT)) break;
                 }
                 tc_fence_after();
-                constexpr int LAST = KW - (UPT - 1) * UW;           // words of the tile's last unit
-                const uint32_t taddr = t_lane + (uint32_t)(ust * C::U_COLS);
-                if (h < UPT - 1) store_words<UW>(taddr, &wds[h * UW]);
-                else store_words<LAST>(taddr, &wds[(UPT - 1) * UW]);
+                const int ast = n % NA;
+                const uint32_t taddr = t_lane + (uint32_t)(ast * C::A_COLS + 8 * T0 * CW);
+                tc_st32_nowait(taddr, v);
+#pragma unroll
+                for (int e4 = 4; e4 + 4 <= W; e4 += 4) {
+                    uint32_t v4[32];
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) expand_a(wds[e4 + e], &v4[8 * e]);
+                    tc_st32_nowait(taddr + 8u * e4, v4);
+                }
+#pragma unroll
+                for (int e = W / 4 * 4; e < W; ++e) {
+                    uint32_t v8[8];
+                    expand_a(wds[e], v8);
+                    tc_st8_nowait(taddr + 8u * e, v8);
+                }
                 tc_wait_st();
                 tc_fence_before();
                 __syncwarp();
-                mbar_arrive_pred(a_full(slot, ust), lane0);
-                ++units;
-                if (++ust == NU) { ust = 0; uphase ^= 1u; }
+                mbar_arrive_pred(a_full(ast), lane0);
             }
+        };
+        if constexpr (C::COOP) {
+            if (grp == 0) produce(std::integral_constant<int, 0>{}, std::integral_constant<int, TAP_SPLIT>{}, 0, 1);
+            else produce(std::integral_constant<int, TAP_SPLIT>{}, std::integral_constant<int, 9>{}, 0, 1);
+        } else {
+            produce(std::integral_constant<int, 0>{}, std::integral_constant<int, 9>{}, grp, NGRP);
         }
     }
 

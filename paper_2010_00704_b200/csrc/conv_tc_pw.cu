@@ -97,12 +97,6 @@ template <int KW, int BN> struct PwCfg {
     static constexpr int SMEM_ASK = SMEM < 120 * 1024 ? 120 * 1024 : SMEM;     // one CTA per SM (it takes all of tensor memory)
 };
 
-// Accumulator column c of a 32-column block holds this channel of the block (see the epilogue's bit gathering).
-__host__ __device__ constexpr int channel_of_column(int c)
-{
-    return c < 16 ? ((c & 1) ? 8 + (c >> 1) : (c >> 1)) : ((c & 1) ? 24 + ((c - 16) >> 1) : 16 + ((c - 16) >> 1));
-}
-
 template <int KW, int BN>
 __global__ void __launch_bounds__(PwCfg<KW, BN>::THREADS, 1)
 conv_tc_pw_kernel(const ConvProblem p)

@@ -53,11 +53,12 @@ __device__ __forceinline__ void pin_regs(uint32_t (&v)[32])
 // Bounded by elapsed clock cycles (about two seconds), checked every 64 polls together with the CTA's abort flag.
 constexpr long long PW_WAIT_CYCLES = 4000000000LL;
 constexpr uint32_t PW_SLEEP_NS = 32;
+template <uint32_t SLEEP = PW_SLEEP_NS>
 static __device__ __noinline__ bool pw_wait_slow(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *err, int code)
 {
     const long long t0 = clock64();
     for (uint32_t it = 1;; ++it) {
-        __nanosleep(PW_SLEEP_NS);
+        __nanosleep(SLEEP);
         if (mbar_try_wait(bar, parity)) return true;
         if ((it & 63u) == 0u) {
             if (*abort_flag) return false;
@@ -68,12 +69,14 @@ static __device__ __noinline__ bool pw_wait_slow(uint32_t bar, uint32_t parity, 
     if (err) atomicCAS(err, 0, code);
     return false;
 }
-// whole-warp wait (every lane polls; the verdict is a vote)
+// whole-warp wait (every lane polls; the verdict is a vote).  SLEEP: nanoseconds between polls - short for hand-overs on
+// a pipeline's critical path, longer for roles with slack (a polling warp takes issue slots from the warps that work).
+template <uint32_t SLEEP = PW_SLEEP_NS>
 __device__ __forceinline__ bool pw_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag, int *err, int code)
 {
     bool ok = mbar_try_wait(bar, parity);
     if (__all_sync(0xffffffffu, ok)) return true;
-    if (!ok) ok = pw_wait_slow(bar, parity, abort_flag, err, code);
+    if (!ok) ok = pw_wait_slow<SLEEP>(bar, parity, abort_flag, err, code);
     return __all_sync(0xffffffffu, ok);
 }
 
@@ -89,6 +92,12 @@ __device__ __forceinline__ uint32_t sign_word(const uint32_t *r)
         w |= ~d & (0x01010101u << s);
     }
     return w;
+}
+
+// Accumulator column c of a 32-column block holds this channel of the block (the order sign_word gathers bits in).
+__host__ __device__ constexpr int channel_of_column(int c)
+{
+    return c < 16 ? ((c & 1) ? 8 + (c >> 1) : (c >> 1)) : ((c & 1) ? 24 + ((c - 16) >> 1) : 16 + ((c - 16) >> 1));
 }
 
 // 32 accumulator columns (32-bit) of this warp's 32 rows, without the completion wait.

@@ -17,7 +17,7 @@ def bk():
     return binding
 
 
-ENGINES = ["auto", "lop3", "mma_b1", "tc_i8", "mma_s8", "tc_ws", "tc_pw"]
+ENGINES = ["auto", "lop3", "mma_b1", "tc_i8", "mma_s8", "tc_ws", "tc_pw", "tc_c3"]
 
 
 def dev(a):
@@ -97,6 +97,13 @@ CONV_SHAPES = [
     (1, 97, 101, 96, 96, 1, 1, 1, 0),      # ... three words of K, 96 of 128 accumulator columns used
     (1, 55, 77, 32, 128, 1, 1, 1, 0),      # ... narrow K, wide N
     (1, 66, 51, 128, 32, 1, 1, 1, 0),      # ... wide K, narrow N
+    (3, 37, 44, 32, 32, 3, 3, 1, 1),       # halo-tile 3x3 engine: 8 x 16 output tiles, ragged in both directions
+    (2, 61, 52, 32, 64, 3, 3, 2, 1),       # ... stride 2, packed 16-bit epilogue with two output words
+    (2, 45, 30, 64, 64, 3, 3, 1, 1),       # ... two-word pixels: both producer groups fill every tile
+    (1, 70, 66, 64, 32, 3, 3, 2, 0),       # ... stride 2 without padding
+    (1, 50, 40, 32, 96, 3, 3, 1, 0),       # ... 96 of 128 accumulator columns, no padding
+    (1, 41, 48, 64, 128, 3, 3, 2, 1),      # ... two-word pixels, 128 channels: one accumulator
+    (1, 30, 34, 64, 64, 3, 3, 1, 1),       # ... image rows of 68 words: W * C_in / 32 is a multiple of 4, W is not
 ]
 
 
@@ -160,12 +167,51 @@ def test_conv_constant_inputs(bk, engine):
     K = 9 * Ci
     xm = -np.ones((B, H, W, Ci), np.int8)
     wp = np.ones((Co, 3, 3, Ci), np.int8)
-    if engine == "tc_pw":
-        pytest.skip("the pointwise engine takes 1x1 layers with packed output only")
+    if engine in ("tc_pw", "tc_c3"):
+        pytest.skip("the pointwise and halo-tile engines have packed output only")
     assert np.all(run_conv(bk, xm, wp, None, 1, 1, engine) == -K)
     assert np.all(run_conv(bk, xm, -wp, None, 2, 1, engine) == K)
     y = run_conv(bk, -xm, wp, None, 1, 1, engine)[0, :, :, 0]
     assert y[4, 4] == K and y[0, 4] == K - 6 * Ci and y[0, 0] == K - 10 * Ci
+
+
+@pytest.mark.parametrize("shape", [
+    (8, 160, 176, 32, 32, 1, 1),      # 1760 tiles: twelve per CTA - every ring (halo tiles, activation stages, "done" barriers) wraps
+    (6, 161, 180, 32, 64, 2, 1),      # stride 2, ragged: 81 x 90 outputs
+    (16, 128, 128, 64, 64, 1, 1),     # two-word pixels, 2048 tiles
+    (7, 100, 90, 64, 32, 2, 0),       # ... stride 2, no padding (image rows of 180 words)
+])
+def test_tc_c3_many_tiles_sampled(bk, oracle, shape):
+    """The halo-tile 3x3 engine over many tiles per CTA, against the oracle at sampled output pixels (image corners and
+    borders, the pixels around tile borders, and random ones) and against the weight-stationary engine everywhere."""
+    B, H, W, Ci, Co, s, p = shape
+    rng = np.random.default_rng(77 + sum(shape))
+    x = synth.pm1(rng, (B, H, W, Ci))
+    w = synth.pm1(rng, (Co, 3, 3, Ci))
+    K = 9 * Ci
+    OH, OW = bk.out_hw(H, W, 3, 3, s, p)
+    thr = plant_extreme_thresholds(synth.thresholds(rng, K, Co), K)
+    xb, wb, dthr = dev(synth.pack_bits(x)), dev(synth.pack_bits(w)), dev(thr)
+    n = B * OH * OW * Co // 8
+    raw, buf = guard_alloc(n)
+    bk.bcnn_conv2d_b1_fused(xb, wb, dthr, buf, B, H, W, Ci, Co, 3, 3, s, p, engine=bk.ENGINES["tc_c3"])
+    torch.cuda.synchronize()
+    assert bk.bcnn_device_error() == 0
+    check_guards(raw, n)
+    got = synth.unpack_bits(buf.cpu().numpy().reshape(B * OH * OW, Co // 8))
+    pix = set()
+    for b in (0, B // 2, B - 1):
+        for oh in (0, 1, 7, 8, 9, OH // 2, OH - 9, OH - 2, OH - 1):
+            for ow in (0, 1, 15, 16, 17, OW // 2, OW - 17, OW - 2, OW - 1):
+                pix.add((b * OH + oh) * OW + ow)
+    pix.update(int(v) for v in rng.integers(0, B * OH * OW, 3000))
+    pix = np.array(sorted(pix), dtype=np.int64)
+    want = oracle.threshold(oracle.conv2d_pixels(x, w, pix, s, p), thr)
+    assert np.array_equal(got[pix], want)
+    ref = torch.zeros(n, dtype=torch.uint8, device="cuda")
+    bk.bcnn_conv2d_b1_fused(xb, wb, dthr, ref, B, H, W, Ci, Co, 3, 3, s, p, engine=bk.ENGINES["tc_ws"])
+    torch.cuda.synchronize()
+    assert torch.equal(ref, buf)                       # (the other engine is itself checked against the oracle above)
 
 
 GEMM_SHAPES = [(1024, 1024, 512), (1024, 1024, 2304), (300, 200, 96), (129, 33, 1056), (64, 512, 4608), (1, 32, 32)]
