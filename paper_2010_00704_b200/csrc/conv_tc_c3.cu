@@ -14,30 +14,32 @@
 // Arithmetic as in the pointwise engine (conv_tc_pw.cu): unsigned activation bytes {0, 2^j} against signed weight bytes,
 // every product +-64, the per-channel constant written by a first MMA against a constant activation tile.
 //
-// One MMA stream, one commit per tile.  Tensor memory holds NACC accumulators and a ring of NA activation tiles (72
-// columns per 32 input channels).  One issuer warp walks the CTA's tiles in order: it waits until the tile's activations
-// are full and its accumulator free, issues the tile's MMAs and ONE commit on the tile's "done" barrier, which both the
-// epilogue (accumulator ready) and the producers (activation stage free again) wait on: a tcgen05.commit costs the
-// issuing thread about a hundred cycles, and a wait on a barrier that is already complete almost nothing, so with the
-// producers ahead the MMAs of consecutive tiles queue back to back.  Two loader warps and two epilogue groups take
-// alternate tiles.  C_in = 64: both producer groups (four warps each) work on EVERY tile - group 0 expands taps 0..4,
-// group 1 taps 5..8 of the same 128 pixels - which halves the time a tile takes to fill; with only two or three
-// activation tiles in tensor memory that time matters.  C_in = 32: the producer groups take alternate tiles (fewer
-// instructions per tile), and so do two issuer warps: there a tile's MMAs take 160 - 320 cycles and one issuer's
-// waits and commit would be the bound.
-// The "done" barriers form a ring of NB = 8 (tile n -> barrier n % 8): a multiple of NACC and at least NA, so that
-// neither waiter can be lapped.
-// K = 288 or 576 makes |accumulator| exceed 16 bits, so the epilogue reads 32-bit accumulators and shifts sign bits in.
+// One commit per tile.  Tensor memory holds NACC accumulators and a ring of NUNIT activation UNITS: the nine taps of
+// 32 input channels of one tile (72 columns).  A tile is one unit for C_in = 32 and two for C_in = 64 (K order: channel
+// word, then tap).  An issuer warp walks tiles in order: it waits until the tile's units are full and its accumulator
+// free, issues the tile's MMAs and ONE commit on the tile's "done" barrier, which the epilogue (accumulator ready) and
+// the producers (units free again) wait on: with the producers ahead the MMAs of consecutive tiles queue back to back.
+// Four producer groups of four warps fill ONE unit of every tile they take:
+//   * C_in = 64 (tiles of 640+ tensor-pipe cycles, one issuer): groups 2 j and 2 j + 1 fill the two units of the tiles
+//     n = j (mod 2).  The ring holds five (six) units = two and a half (three) tiles, so a tile's first unit reuses
+//     columns that were free one tile earlier than those of its second unit: only half of a tile's stores have to fit
+//     into the time of one tile's MMAs;
+//   * C_in = 32 (tiles of 160 - 320 tensor-pipe cycles, bound by instruction issue): group j fills the tiles
+//     n = j (mod 4), and two issuer warps take alternate tiles (one issuer's waits and commit would be the bound); the
+//     ring then has an even number of units, so that a unit's next user belongs to the same issuer.
+// Two loader warps and two epilogue groups take alternate tiles.
+// The "done" barriers form a ring of NB = 8 (tile n -> barrier n % 8), a multiple of NACC and more than the tiles in
+// flight.  K = 288: |accumulator| <= 32 (2 K + 1) < 2^15, so the epilogue reads packed 16-bit halves and gathers sign
+// bits with byte permutes; K = 576: 32-bit accumulators, sign bits shifted in.
 // A parity wait on an mbarrier is only right while the waiter starts waiting for completion k after completion k - 1 and
 // before completion k + 1.  Tile n's "done" is completion n / 8 of its barrier; its waiters are the epilogue of tile n
-// and the producers of tile n + NA.  Both have seen tile n - 2 done (an issuer's tiles complete in order: so is tile
-// n - 8), and tile n + 8 cannot be issued before both are through: its issuer first issues tile n + NA (the same
-// issuer: NA is a multiple of the number of issuers), which needs that tile's activations, and, NB being a multiple
-// of NACC, tile n + 8 needs the accumulator of tile n back from the epilogue.
+// and the producers of the tiles (at most four ahead) that reuse its units.  Every one of them has seen an earlier tile
+// of the same issuer done within the last eight (an issuer's tiles complete in order), and tile n + 8 cannot be issued
+// before they are through: its issuer first issues the reusing tiles (the same issuer), which need those units filled,
+// and, NB being a multiple of NACC, tile n + 8 needs the accumulator of tile n back from the epilogue.
 // Every mbarrier wait is bounded and reports through the device error word.
 #include "tc_slot.cuh"
 #include <cuda.h>
-#include <type_traits>
 
 namespace bcnn {
 
@@ -49,44 +51,41 @@ constexpr int ERR_C3_LOADER_TIMEOUT = 141;       // loader: no free ring stage
 constexpr int ERR_C3_PRODUCER_TIMEOUT = 142;     // producer: the tile's halo did not arrive
 constexpr int ERR_C3_ISSUER_TIMEOUT = 143;       // issuer: a tile's activations were not filled
 constexpr int ERR_C3_EPILOGUE_TIMEOUT = 144;     // epilogue: the tile's MMAs did not complete
-constexpr int ERR_C3_UNIT_TIMEOUT = 145;         // producer: the activation stage's previous MMAs did not complete
+constexpr int ERR_C3_UNIT_TIMEOUT = 145;         // producer: the unit's previous MMAs did not complete
 constexpr int ERR_C3_ACC_TIMEOUT = 146;          // issuer: an accumulator was not handed back
 
 constexpr int TH = 8, TW = 16;            // output tile (TH * TW = 128 = tensor-memory lanes)
-constexpr int NGRP = 2;                   // loader / epilogue groups (alternate tiles); producer groups (taps 0..4 / 5..8 of every tile)
-constexpr int TAP_SPLIT = 5;
-constexpr int RD = 6;                     // halo tiles in a group's ring
+constexpr int NGRP = 2;                   // loader / epilogue groups (alternate tiles)
+constexpr int NPG = 4;                    // producer groups of four warps
+constexpr int RD = 6;                     // halo tiles in a loader's ring
 constexpr int CONST_COLS = 8;
+constexpr int TAPS = 9;
+constexpr int U_COLS = 8 * TAPS;          // columns of a unit
 constexpr int NB = 8;                     // ring of "tile done" barriers
-constexpr int MAX_NA = 5, MAX_NACC = 4;
+constexpr int NAF = 4;                    // ring of "tile full" barriers (at most four tiles are being filled)
+constexpr int MAX_NUNIT = 6, MAX_NACC = 4;
 
 // CW: words per input pixel (1, 2) = units per tile; BN: accumulator columns per tile (32, 64, 128 >= C_out).
 template <int CW, int BN> struct C3Cfg {
-    static constexpr int KW = 9 * CW;                       // words of K per row
+    static constexpr int KW = TAPS * CW;                    // words of K per row
     static constexpr int KT = (KW + 3) / 4;                 // 128-byte stages of the expanded weights
-    static constexpr int A_COLS = 8 * KW;                   // columns of one activation tile
     static constexpr int NACC = CW == 2 && BN == 128 ? 1 : (CW == 1 && BN == 32 ? 4 : 2);   // accumulators
-    static constexpr int NA0 = (512 - CONST_COLS - NACC * BN) / A_COLS;
-    // C_in = 64 (MMA-bound tiles): one issuer; both producer groups fill every tile (COOP).  C_in = 32 (short tiles, bound
-    // by instruction issue): two issuer warps and the producer groups take alternate tiles; then a tile and the next user
-    // of its activation stage must belong to the same issuer, so the ring has an even number of stages.
-    static constexpr bool COOP = CW == 2;
-    // K = 288: |accumulator| <= 32 (2 K + 1) < 2^15, so the epilogue can read packed 16-bit halves and gather sign bits
-    // with byte permutes (half the logic operations); the weight rows are then laid out in the gathering's column order
+    static constexpr int NISS = CW == 2 ? 1 : 2;            // issuer warps
     static constexpr bool PACK16 = CW == 1;
-    static constexpr int NISS = CW == 2 ? 1 : 2;
-    static constexpr int NA1 = NA0 > MAX_NA ? MAX_NA : NA0;
-    static constexpr int NA = NISS == 2 ? NA1 / 2 * 2 : NA1;   // activation tiles in the ring: 4, 4, 2 (C_in 32); 3, 2, 2 (C_in 64)
+    static constexpr int NU0 = (512 - CONST_COLS - NACC * BN) / U_COLS;
+    static constexpr int NU1 = NU0 > MAX_NUNIT ? MAX_NUNIT : NU0;
+    static constexpr int NUNIT = CW == 1 ? (NU1 > 4 ? 4 : NU1 / 2 * 2) : NU1;   // 4, 4, 2 (C_in 32); 6, 5, 5 (C_in 64)
     static constexpr int A_COL0 = NACC * BN;
-    static constexpr int C_COL = A_COL0 + NA * A_COLS;      // the constant activation tile
+    static constexpr int C_COL = A_COL0 + NUNIT * U_COLS;   // the constant activation tile
     static_assert(C_COL + CONST_COLS <= 512, "tensor memory budget");
-    static_assert(NA >= 2 && NA <= NB && NB % NACC == 0 && NACC <= MAX_NACC && NACC % NISS == 0 && NA % NISS == 0, "barrier rings");
-    // warps: 0 (and 1) issuers, 2 and 3 loaders, then per group four producer warps, then per group four epilogue
-    // warps (groups start at multiples of four: warp % 4 is the tensor-memory lane quadrant of a warp)
+    static_assert(NUNIT >= 2 * CW && (NUNIT + CW - 1) / CW <= NAF && NB % NACC == 0 && NACC <= MAX_NACC && NACC % NISS == 0 &&
+                  (NISS == 1 || NUNIT % NISS == 0), "barrier rings");
+    // warps: 0 (and 1) issuers, 2 and 3 loaders, then the producer groups, then the epilogue groups (groups start at
+    // multiples of four: warp % 4 is the tensor-memory lane quadrant of a warp)
     static constexpr int FIRST_LOADER_WARP = 2;
     static constexpr int FIRST_PRODUCER_WARP = 4;
-    static constexpr int FIRST_EPILOGUE_WARP = 4 + 4 * NGRP;
-    static constexpr int WARPS = 4 + 8 * NGRP;
+    static constexpr int FIRST_EPILOGUE_WARP = 4 + 4 * NPG;
+    static constexpr int WARPS = 4 + 4 * NPG + 4 * NGRP;
     static constexpr int THREADS = 32 * WARPS;
     static constexpr int W_TILE_BYTES = BN * ROWB;
 };
@@ -127,8 +126,8 @@ __global__ void __launch_bounds__(C3Cfg<CW, BN>::THREADS, 1)
 conv_tc_c3_kernel(const ConvProblem p, const C3Geom g, const __grid_constant__ CUtensorMap xmap)
 {
     using C = C3Cfg<CW, BN>;
-    constexpr int KW = C::KW, KT = C::KT, NACC = C::NACC, NA = C::NA;
-    constexpr int NBARS = 2 * NGRP * RD + MAX_NA + NB + MAX_NACC;
+    constexpr int KW = C::KW, KT = C::KT, NACC = C::NACC, NUNIT = C::NUNIT;
+    constexpr int NBARS = 2 * NGRP * RD + NAF + NB + MAX_NACC;
 
     extern __shared__ unsigned char smem_raw[];
     __shared__ __align__(8) unsigned long long bars[NBARS];
@@ -138,7 +137,8 @@ conv_tc_c3_kernel(const ConvProblem p, const C3Geom g, const __grid_constant__ C
     const int tid = threadIdx.x;
     const int warp = tid >> 5, lane = tid & 31;
     // this CTA's tiles: blockIdx.x + n * gridDim.x, n = 0, 1, ...; tile n belongs to loader / epilogue group n % 2, uses
-    // accumulator n % NACC, activation stage n % NA and "done" barrier n % NB
+    // accumulator n % NACC, "full" barrier n % NAF, "done" barrier n % NB; its unit h is the CTA's unit number n * CW + h,
+    // in ring position (n * CW + h) % NUNIT
     const int my_tiles = (int)blockIdx.x < g.total_tiles ? (g.total_tiles - 1 - (int)blockIdx.x) / (int)gridDim.x + 1 : 0;
     const int cn = min(BN, p.C_out);
 
@@ -149,16 +149,16 @@ conv_tc_c3_kernel(const ConvProblem p, const C3Geom g, const __grid_constant__ C
     auto load_full = [&](int gr, int s) { return bar0 + 8u * (gr * RD + s); };
     auto load_empty = [&](int gr, int s) { return bar0 + 8u * (NGRP * RD + gr * RD + s); };
     auto a_full = [&](int s) { return bar0 + 8u * (2 * NGRP * RD + s); };
-    auto tile_done = [&](int s) { return bar0 + 8u * (2 * NGRP * RD + MAX_NA + s); };
-    auto acc_free = [&](int s) { return bar0 + 8u * (2 * NGRP * RD + MAX_NA + NB + s); };
+    auto tile_done = [&](int s) { return bar0 + 8u * (2 * NGRP * RD + NAF + s); };
+    auto acc_free = [&](int s) { return bar0 + 8u * (2 * NGRP * RD + NAF + NB + s); };
     volatile int *abort_flag = &abort_flag_smem;
 
     if (tid == 0) {
         for (int s = 0; s < NGRP * RD; ++s) {
             mbar_init(load_full(0, s), 1);              // the loader's arrive (+ the copy's bytes)
-            mbar_init(load_empty(0, s), C::COOP ? 8 : 4);   // the producer warps that read the stage
+            mbar_init(load_empty(0, s), 4 * CW);        // the producer warps that read the stage
         }
-        for (int s = 0; s < MAX_NA; ++s) mbar_init(a_full(s), C::COOP ? 8 : 4);   // the producer warps that fill the stage
+        for (int s = 0; s < NAF; ++s) mbar_init(a_full(s), 4 * CW);     // the producer warps that fill the tile's units
         for (int s = 0; s < NB; ++s) mbar_init(tile_done(s), 1);        // the issuer's commit
         for (int s = 0; s < MAX_NACC; ++s) mbar_init(acc_free(s), 4);   // the four epilogue warps of the tile's group
         abort_flag_smem = 0;
@@ -168,9 +168,10 @@ conv_tc_c3_kernel(const ConvProblem p, const C3Geom g, const __grid_constant__ C
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_smem)), "r"(512u) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
-    // ---- one-off: expanded weights (K word e -> stage e / 4, 32-byte piece e % 4) and the constant bytes
+    // ---- one-off: expanded weights and the constant bytes.  K position e of the MMAs = channel word e / 9, tap e % 9
+    // (global weight word tap * CW + channel word) -> stage e / 4, 32-byte piece e % 4; MMA row `row` carries channel ch
     for (int idx = tid; idx < (KT + 1) * BN; idx += C::THREADS) {
-        const int kt = idx / BN, row = idx - kt * BN;       // MMA row `row` carries channel ch
+        const int kt = idx / BN, row = idx - kt * BN;
         const int ch = C::PACK16 ? (row & ~31) + channel_of_column(row & 31) : row;
         const bool have = ch < cn;
         const int xr = row & 7;
@@ -178,9 +179,9 @@ conv_tc_c3_kernel(const ConvProblem p, const C3Geom g, const __grid_constant__ C
             const uint32_t row_addr = wexp + (uint32_t)kt * C::W_TILE_BYTES + (uint32_t)row * ROWB;
 #pragma unroll
             for (int e = 0; e < 4; ++e) {
-                const int kword = kt * 4 + e;
-                const bool live = kword < KW && have;
-                const uint32_t w = live ? __ldg(p.w + (long)ch * KW + kword) : 0u;
+                const int kpos = kt * 4 + e;
+                const bool live = kpos < KW && have;
+                const uint32_t w = live ? __ldg(p.w + (long)ch * KW + (kpos % TAPS) * CW + kpos / TAPS) : 0u;
                 expand_store_w_signed(w, live, row_addr, xr, 2 * e);
             }
         } else {
@@ -241,18 +242,23 @@ conv_tc_c3_kernel(const ConvProblem p, const C3Geom g, const __grid_constant__ C
         const uint32_t tmem_u = __shfl_sync(0xffffffffu, tmem_base, 0);
         const uint32_t c_t = tmem_u + (uint32_t)C::C_COL;
         for (int n = warp; n < my_tiles; n += C::NISS) {
-            const int ast = n % NA, acc = n % NACC;
-            if (!pw_wait(a_full(ast), (uint32_t)(n / NA) & 1u, abort_flag, p.err, ERR_C3_ISSUER_TIMEOUT)) break;
+            const int acc = n % NACC;
+            if (!pw_wait(a_full(n % NAF), (uint32_t)(n / NAF) & 1u, abort_flag, p.err, ERR_C3_ISSUER_TIMEOUT)) break;
             // the epilogue has read the accumulator's previous tile
             if (n >= NACC && !pw_wait(acc_free(acc), (uint32_t)(n / NACC - 1) & 1u, abort_flag, p.err, ERR_C3_ACC_TIMEOUT)) break;
             tc_fence_after();
             if (elect_one()) {
                 const uint32_t d_t = tmem_u + (uint32_t)(acc * BN);
-                const uint32_t a_t = tmem_u + (uint32_t)(C::A_COL0 + ast * C::A_COLS);
                 tc_mma_i8_ts(d_t, c_t, c_lo, desc_hi, idesc, 0u);               // accumulator = the per-channel constants
 #pragma unroll
-                for (int e = 0; e < KW; ++e)
-                    tc_mma_i8_ts(d_t, a_t + 8u * e, b_lo + (uint32_t)((e >> 2) * (C::W_TILE_BYTES >> 4) + 2 * (e & 3)), desc_hi, idesc, 1u);
+                for (int h = 0; h < CW; ++h) {
+                    const uint32_t a_t = tmem_u + (uint32_t)(C::A_COL0 + ((n * CW + h) % NUNIT) * U_COLS);
+#pragma unroll
+                    for (int t = 0; t < TAPS; ++t) {
+                        const int e = h * TAPS + t;
+                        tc_mma_i8_ts(d_t, a_t + 8u * t, b_lo + (uint32_t)((e >> 2) * (C::W_TILE_BYTES >> 4) + 2 * (e & 3)), desc_hi, idesc, 1u);
+                    }
+                }
                 tc_commit(tile_done(n % NB));
             }
             __syncwarp();
@@ -262,32 +268,30 @@ conv_tc_c3_kernel(const ConvProblem p, const C3Geom g, const __grid_constant__ C
     } else if (warp < C::FIRST_PRODUCER_WARP) {
         // ------------------------------------------------------------------ loader of group warp - 2: one halo tile per TMA copy
         const int grp = warp - C::FIRST_LOADER_WARP;
-        {
-            int stage = 0;
-            uint32_t phase = 1;                       // first pass through the ring: the stages are free
-            int issued = 0;
-            for (int n = grp; n < my_tiles; n += NGRP) {
-                if (!pw_wait<256>(load_empty(grp, stage), phase, abort_flag, p.err, ERR_C3_LOADER_TIMEOUT)) break;
-                if (lane == 0) {
-                    const uint32_t dst = ring + (uint32_t)(grp * RD + stage) * (uint32_t)g.stage_bytes;
-                    int b, oh0, ow0;
-                    tile_origin(tile_of(n), b, oh0, ow0);
-                    const int x = (ow0 * g.stride - p.pad - g.xoff) * CW;        // words; a multiple of 4 by construction
-                    const int y = oh0 * g.stride - p.pad;
-                    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(load_full(grp, stage)), "r"((uint32_t)(g.hb * g.wbw * 4)) : "memory");
-                    asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
-                                 ::"r"(dst), "l"(reinterpret_cast<uint64_t>(&xmap)), "r"(x), "r"(y), "r"(b), "r"(load_full(grp, stage)) : "memory");
-                }
-                __syncwarp();
-                ++issued;
-                if (++stage == RD) { stage = 0; phase ^= 1u; }
+        int stage = 0;
+        uint32_t phase = 1;                       // first pass through the ring: the stages are free
+        int issued = 0;
+        for (int n = grp; n < my_tiles; n += NGRP) {
+            if (!pw_wait<256>(load_empty(grp, stage), phase, abort_flag, p.err, ERR_C3_LOADER_TIMEOUT)) break;
+            if (lane == 0) {
+                const uint32_t dst = ring + (uint32_t)(grp * RD + stage) * (uint32_t)g.stage_bytes;
+                int b, oh0, ow0;
+                tile_origin(tile_of(n), b, oh0, ow0);
+                const int x = (ow0 * g.stride - p.pad - g.xoff) * CW;        // words; a multiple of 4 by construction
+                const int y = oh0 * g.stride - p.pad;
+                asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(load_full(grp, stage)), "r"((uint32_t)(g.hb * g.wbw * 4)) : "memory");
+                asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+                             ::"r"(dst), "l"(reinterpret_cast<uint64_t>(&xmap)), "r"(x), "r"(y), "r"(b), "r"(load_full(grp, stage)) : "memory");
             }
-            // after a time-out elsewhere: copies still in flight must land before the CTA's shared memory goes away
-            if (*abort_flag) {
-                const int first = issued > RD ? issued - RD : 0;
-                for (int q = first; q < issued; ++q)
-                    pw_wait(load_full(grp, q % RD), (uint32_t)(q / RD) & 1u, abort_flag, nullptr, 0);
-            }
+            __syncwarp();
+            ++issued;
+            if (++stage == RD) { stage = 0; phase ^= 1u; }
+        }
+        // after a time-out elsewhere: copies still in flight must land before the CTA's shared memory goes away
+        if (*abort_flag) {
+            const int first = issued > RD ? issued - RD : 0;
+            for (int q = first; q < issued; ++q)
+                pw_wait(load_full(grp, q % RD), (uint32_t)(q / RD) & 1u, abort_flag, nullptr, 0);
         }
     } else if (warp >= C::FIRST_EPILOGUE_WARP) {
         // ------------------------------------------------------------------ epilogue group (warp - first) / 4
@@ -298,7 +302,7 @@ conv_tc_c3_kernel(const ConvProblem p, const C3Geom g, const __grid_constant__ C
         const int owords = p.C_out >> 5;
         for (int n = grp; n < my_tiles; n += NGRP) {
             const int acc = n % NACC;
-            if (!pw_wait<128>(tile_done(n % NB), (uint32_t)(n / NB) & 1u, abort_flag, p.err, ERR_C3_EPILOGUE_TIMEOUT)) break;
+            if (!pw_wait<C::NISS == 1 ? 64 : 128>(tile_done(n % NB), (uint32_t)(n / NB) & 1u, abort_flag, p.err, ERR_C3_EPILOGUE_TIMEOUT)) break;
             tc_fence_after();
             uint32_t words[BN / 32];
             if constexpr (C::PACK16) {
@@ -328,26 +332,26 @@ conv_tc_c3_kernel(const ConvProblem p, const C3Geom g, const __grid_constant__ C
                 }
             } else {
 #pragma unroll
-            for (int ch = 0; ch < BN / 32; ++ch) {
-                words[ch] = 0;
-                if (ch * 32 < cn) {                                   // warp-uniform
-                    uint32_t v[32];
-                    tc_ld32(t_lane + (uint32_t)(acc * BN + ch * 32), v);
-                    if ((ch + 1) * 32 >= cn) {                        // the accumulator's last columns are in registers
-                        tc_fence_before();
-                        __syncwarp();
-                        if (lane == 0) mbar_arrive(acc_free(acc));
-                    }
-                    // bit i = (v[i] >= 0): sign bits shifted in, last column first; two chains of 16
-                    uint32_t hi = 0, lo = 0;
+                for (int ch = 0; ch < BN / 32; ++ch) {
+                    words[ch] = 0;
+                    if (ch * 32 < cn) {                                   // warp-uniform
+                        uint32_t v[32];
+                        tc_ld32(t_lane + (uint32_t)(acc * BN + ch * 32), v);
+                        if ((ch + 1) * 32 >= cn) {                        // the accumulator's last columns are in registers
+                            tc_fence_before();
+                            __syncwarp();
+                            if (lane == 0) mbar_arrive(acc_free(acc));
+                        }
+                        // bit i = (v[i] >= 0): sign bits shifted in, last column first; two chains of 16
+                        uint32_t hi = 0, lo = 0;
 #pragma unroll
-                    for (int i = 15; i >= 0; --i) {
-                        hi = __funnelshift_l(v[16 + i], hi, 1);
-                        lo = __funnelshift_l(v[i], lo, 1);
+                        for (int i = 15; i >= 0; --i) {
+                            hi = __funnelshift_l(v[16 + i], hi, 1);
+                            lo = __funnelshift_l(v[i], lo, 1);
+                        }
+                        words[ch] = ~__byte_perm(lo, hi, 0x5410);
                     }
-                    words[ch] = ~__byte_perm(lo, hi, 0x5410);
                 }
-            }
             }
             int b, oh0, ow0;
             tile_origin(tile_of(n), b, oh0, ow0);
@@ -368,71 +372,53 @@ conv_tc_c3_kernel(const ConvProblem p, const C3Geom g, const __grid_constant__ C
     } else {
         // ------------------------------------------------------------------ producer group (warp - first) / 4
         // thread = output pixel (ty, tx) of the tile = tensor-memory lane; its nine input pixels sit at rows
-        // ty * s + kr, pixels tx * s + XOFF + kt of the halo tile.  K word order: tap-major (tap = 3 kr + kt), the
-        // pixel's words within a tap.  Group 0 takes taps 0..4, group 1 taps 5..8 of every tile.
+        // ty * s + kr, pixels tx * s + XOFF + kt of the halo tile.  The group fills unit h (channel word h of the nine
+        // taps) of the tiles n0, n0 + step, ...
         const int quad = warp & 3;
         const int grp = (warp - C::FIRST_PRODUCER_WARP) >> 2;
+        const int h = CW == 2 ? (grp & 1) : 0;
+        const int n0 = CW == 2 ? (grp >> 1) : grp, step = CW == 2 ? NPG / 2 : NPG;
         const int r = quad * 32 + lane;
-        const uint32_t my_off = (uint32_t)((((r >> 4) * g.stride) * g.wbw + ((r & 15) * g.stride + g.xoff) * CW) * 4);
+        const uint32_t my_off = (uint32_t)((((r >> 4) * g.stride) * g.wbw + ((r & 15) * g.stride + g.xoff) * CW + h) * 4);
         const uint32_t row_pitch = (uint32_t)(g.wbw * 4);
         const uint32_t t_lane = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)C::A_COL0;
         const uint32_t lane0 = lane == 0 ? 1u : 0u;
-        // taps [T0, T1) of every tile: W = (T1 - T0) * CW words, tensor-memory columns from 8 * T0 * CW of the stage
-        auto produce = [&](auto t0c, auto t1c, const int n0, const int step) {
-            constexpr int T0 = decltype(t0c)::value, T1 = decltype(t1c)::value, W = (T1 - T0) * CW;
-            for (int n = n0; n < my_tiles; n += step) {
-                const int lg = n & 1, stage = (n >> 1) % RD;
-                uint32_t wds[W];
-                if (!pw_wait<64>(load_full(lg, stage), (uint32_t)((n >> 1) / RD) & 1u, abort_flag, p.err, ERR_C3_PRODUCER_TIMEOUT)) break;
-                const uint32_t src = ring + (uint32_t)(lg * RD + stage) * (uint32_t)g.stage_bytes + my_off;
+        for (int n = n0; n < my_tiles; n += step) {
+            const int lg = n & 1, stage = (n >> 1) % RD;
+            uint32_t wds[TAPS];
+            if (!pw_wait<64>(load_full(lg, stage), (uint32_t)((n >> 1) / RD) & 1u, abort_flag, p.err, ERR_C3_PRODUCER_TIMEOUT)) break;
+            const uint32_t src = ring + (uint32_t)(lg * RD + stage) * (uint32_t)g.stage_bytes + my_off;
 #pragma unroll
-                for (int tap = T0; tap < T1; ++tap) {
-                    const uint32_t a = src + (uint32_t)(tap / 3) * row_pitch + (uint32_t)((tap % 3) * CW * 4);
-                    if constexpr (CW == 2) {
-                        asm volatile("ld.shared.v2.b32 {%0,%1}, [%2];" : "=r"(wds[(tap - T0) * 2]), "=r"(wds[(tap - T0) * 2 + 1]) : "r"(a) : "memory");
-                    } else {
-                        asm volatile("ld.shared.b32 %0, [%1];" : "=r"(wds[tap - T0]) : "r"(a) : "memory");
-                    }
-                }
-                __syncwarp();
-                mbar_arrive_pred(load_empty(lg, stage), lane0);        // the stage may be refilled
-                // the first four words are expanded before the wait for the activation stage
-                uint32_t v[32];
+            for (int tap = 0; tap < TAPS; ++tap)
+                asm volatile("ld.shared.b32 %0, [%1];" : "=r"(wds[tap]) : "r"(src + (uint32_t)(tap / 3) * row_pitch + (uint32_t)((tap % 3) * CW * 4)) : "memory");
+            __syncwarp();
+            mbar_arrive_pred(load_empty(lg, stage), lane0);        // the stage may be refilled
+            // the first four words are expanded before the wait for the unit
+            uint32_t v[32];
 #pragma unroll
-                for (int e = 0; e < 4; ++e) expand_a(wds[e], &v[8 * e]);
-                // the MMAs of tile n - NA have read the stage (nothing to wait for the first time round the ring)
-                if (n >= NA) {
-                    const int m = n - NA;
-                    if (!pw_wait<64>(tile_done(m % NB), (uint32_t)(m / NB) & 1u, abort_flag, p.err, ERR_C3_UNIT_TIMEOUT)) break;
-                }
-                tc_fence_after();
-                const int ast = n % NA;
-                const uint32_t taddr = t_lane + (uint32_t)(ast * C::A_COLS + 8 * T0 * CW);
-                tc_st32_nowait(taddr, v);
-#pragma unroll
-                for (int e4 = 4; e4 + 4 <= W; e4 += 4) {
-                    uint32_t v4[32];
-#pragma unroll
-                    for (int e = 0; e < 4; ++e) expand_a(wds[e4 + e], &v4[8 * e]);
-                    tc_st32_nowait(taddr + 8u * e4, v4);
-                }
-#pragma unroll
-                for (int e = W / 4 * 4; e < W; ++e) {
-                    uint32_t v8[8];
-                    expand_a(wds[e], v8);
-                    tc_st8_nowait(taddr + 8u * e, v8);
-                }
-                tc_wait_st();
-                tc_fence_before();
-                __syncwarp();
-                mbar_arrive_pred(a_full(ast), lane0);
+            for (int e = 0; e < 4; ++e) expand_a(wds[e], &v[8 * e]);
+            // the MMAs of the tile that used this ring position last have read it (nothing to wait for the first time round)
+            const int u = n * CW + h;
+            if (u >= NUNIT) {
+                const int m = (u - NUNIT) / CW;
+                if (!pw_wait<64>(tile_done(m % NB), (uint32_t)(m / NB) & 1u, abort_flag, p.err, ERR_C3_UNIT_TIMEOUT)) break;
             }
-        };
-        if constexpr (C::COOP) {
-            if (grp == 0) produce(std::integral_constant<int, 0>{}, std::integral_constant<int, TAP_SPLIT>{}, 0, 1);
-            else produce(std::integral_constant<int, TAP_SPLIT>{}, std::integral_constant<int, 9>{}, 0, 1);
-        } else {
-            produce(std::integral_constant<int, 0>{}, std::integral_constant<int, 9>{}, grp, NGRP);
+            tc_fence_after();
+            const uint32_t taddr = t_lane + (uint32_t)((u % NUNIT) * U_COLS);
+            tc_st32_nowait(taddr, v);
+            {
+                uint32_t v4[32];
+#pragma unroll
+                for (int e = 0; e < 4; ++e) expand_a(wds[4 + e], &v4[8 * e]);
+                tc_st32_nowait(taddr + 32u, v4);
+                uint32_t v8[8];
+                expand_a(wds[8], v8);
+                tc_st8_nowait(taddr + 64u, v8);
+            }
+            tc_wait_st();
+            tc_fence_before();
+            __syncwarp();
+            mbar_arrive_pred(a_full(n % NAF), lane0);
         }
     }
 
