@@ -316,8 +316,9 @@ def bound_and_frac(ops: float, nbytes: float, ms: float, tensor_peak: float, hbm
 
 
 def other_configs(tensor_peak: float, hbm_gbs: float, steps: int = 20, warmup: int = 5):
-    """The other benchmark workloads (single 3x3 layer, GEMM sweep int32 + fused, stem / down-sampling layers, block
-    stack), AUTO engine, 20 launches each with L2 flushed in between: median and min time, TOP/s and the fraction of
+    """The other benchmark workloads (single 3x3 layer, GEMM sweep int32 + fused - plain calls and the calls on
+    prepared weights -, stem / down-sampling layers, block stack), AUTO engine, 20 launches each with L2 flushed in
+    between: median and min time, TOP/s and the fraction of
     the bounding roof (tensor pipe or HBM, on algorithmic bytes: packed inputs + weights + output)."""
     import torch
     from paper_2010_00704_b200 import binding
@@ -360,7 +361,14 @@ def other_configs(tensor_peak: float, hbm_gbs: float, steps: int = 20, warmup: i
             add(f"gemm M=N={M} K={k} int32", lambda: binding.bcnn_gemm_b1(A, Wb, out32, M, N, k), ops, (M + N) * k // 8 + 4 * M * N)
             add(f"gemm M=N={M} K={k} fused", lambda: binding.bcnn_gemm_b1_fused(A, Wb, thr, outb, M, N, k), ops,
                 (M + N) * k // 8 + M * N // 8)
-            del A, Wb, thr, out32, outb
+            # the same products on prepared weights (expanded once by bcnn_prepare_weights, outside the timed call)
+            prep = torch.empty(binding.bcnn_prepared_weights_bytes(N, k), dtype=torch.uint8, device="cuda")
+            binding.bcnn_prepare_weights(Wb, prep, N, k)
+            add(f"gemm M=N={M} K={k} int32, prepared weights", lambda: binding.bcnn_gemm_b1_prepared(A, prep, None, out32, M, N, k),
+                ops, (M + N) * k // 8 + 4 * M * N)
+            add(f"gemm M=N={M} K={k} fused, prepared weights", lambda: binding.bcnn_gemm_b1_prepared(A, prep, thr, outb, M, N, k),
+                ops, (M + N) * k // 8 + M * N // 8)
+            del A, Wb, thr, out32, outb, prep
     for l in wl.STEM_DOWN:
         conv_case("stem/down:", l, wl.STEM_DOWN_BATCH)
     for l in wl.BLOCK_STACK:
