@@ -553,7 +553,10 @@ def run_gpu(args):
     # the roofline entry describes the dominant kernel's costliest launch: algorithmic ops of that
     # layer / its average launch duration (CUDA events around each launch, averaged over the steps)
     dom_engine = [e for e in kernel_of if kernel_of[e] == groups[0]["kernel"]][0]
-    top = max((i for i, e in enumerate(engines) if e == dom_engine), key=lambda i: per_ms[i + 1])
+    # (layers of equal shape time within noise of each other: the first one within 7 % of the slowest stands for them)
+    dom_idx = [i for i, e in enumerate(engines) if e == dom_engine]
+    slowest = max(per_ms[i + 1] for i in dom_idx)
+    top = next(i for i in dom_idx if per_ms[i + 1] >= 0.93 * slowest)
     lt = layers[top]
     top_tops = lt.ops(B) / (per_ms[top + 1] / 1e3) / 1e12
     src_of = {"tc_ws": ["conv_tc_ws.cu", "tc_common.cuh"], "tc_i8": ["conv_tc_i8.cu", "tc_common.cuh"],
