@@ -69,13 +69,18 @@ constexpr int MAX_NUNIT = 6, MAX_NACC = 4;
 template <int CW, int BN> struct C3Cfg {
     static constexpr int KW = TAPS * CW;                    // words of K per row
     static constexpr int KT = (KW + 3) / 4;                 // 128-byte stages of the expanded weights
-    static constexpr int NACC = CW == 2 && BN == 128 ? 1 : (CW == 1 && BN == 32 ? 4 : 2);   // accumulators
-    static constexpr int NISS = CW == 2 ? 1 : 2;            // issuer warps
+    // 128 output channels run as two halves of 64 against the same activation units: the accumulator of one half is
+    // read by its epilogue group while the other half's MMAs run (one 128-column accumulator would leave room for
+    // neither a second one nor enough units)
+    static constexpr int NH = BN == 128 ? 2 : 1;            // halves
+    static constexpr int AW = BN / NH;                      // accumulator columns
+    static constexpr int NACC = NH == 2 ? 2 : (CW == 1 && BN == 32 ? 4 : 2);   // accumulators (NH == 2: one per half)
+    static constexpr int NISS = CW == 2 || NH == 2 ? 1 : 2; // issuer warps
     static constexpr bool PACK16 = CW == 1;
-    static constexpr int NU0 = (512 - CONST_COLS - NACC * BN) / U_COLS;
+    static constexpr int NU0 = (512 - CONST_COLS - NACC * AW) / U_COLS;
     static constexpr int NU1 = NU0 > MAX_NUNIT ? MAX_NUNIT : NU0;
-    static constexpr int NUNIT = CW == 1 ? (NU1 > 4 ? 4 : NU1 / 2 * 2) : NU1;   // 4, 4, 2 (C_in 32); 6, 5, 5 (C_in 64)
-    static constexpr int A_COL0 = NACC * BN;
+    static constexpr int NUNIT = CW == 1 ? (NU1 > 4 ? 4 : NU1 / 2 * 2) : NU1;   // 4 (C_in 32); 6, 5, 5 (C_in 64)
+    static constexpr int A_COL0 = NACC * AW;
     static constexpr int C_COL = A_COL0 + NUNIT * U_COLS;   // the constant activation tile
     static_assert(C_COL + CONST_COLS <= 512, "tensor memory budget");
     static_assert(NUNIT >= 2 * CW && (NUNIT + CW - 1) / CW <= NAF && NB % NACC == 0 && NACC <= MAX_NACC && NACC % NISS == 0 &&
@@ -126,7 +131,7 @@ __global__ void __launch_bounds__(C3Cfg<CW, BN>::THREADS, 1)
 conv_tc_c3_kernel(const ConvProblem p, const C3Geom g, const __grid_constant__ CUtensorMap xmap)
 {
     using C = C3Cfg<CW, BN>;
-    constexpr int KW = C::KW, KT = C::KT, NACC = C::NACC, NUNIT = C::NUNIT;
+    constexpr int KW = C::KW, KT = C::KT, NACC = C::NACC, NUNIT = C::NUNIT, NH = C::NH, AW = C::AW;
     constexpr int NBARS = 2 * NGRP * RD + NAF + NB + MAX_NACC;
 
     extern __shared__ unsigned char smem_raw[];
@@ -137,7 +142,8 @@ conv_tc_c3_kernel(const ConvProblem p, const C3Geom g, const __grid_constant__ C
     const int tid = threadIdx.x;
     const int warp = tid >> 5, lane = tid & 31;
     // this CTA's tiles: blockIdx.x + n * gridDim.x, n = 0, 1, ...; tile n belongs to loader / epilogue group n % 2, uses
-    // accumulator n % NACC, "full" barrier n % NAF, "done" barrier n % NB; its unit h is the CTA's unit number n * CW + h,
+    // accumulator n % NACC, "full" barrier n % NAF, "done" barrier n % NB (two halves: both epilogue groups, accumulator =
+    // half, "done" barrier (2 n + half) % NB); its unit h is the CTA's unit number n * CW + h,
     // in ring position (n * CW + h) % NUNIT
     const int my_tiles = (int)blockIdx.x < g.total_tiles ? (g.total_tiles - 1 - (int)blockIdx.x) / (int)gridDim.x + 1 : 0;
     const int cn = min(BN, p.C_out);
@@ -235,33 +241,43 @@ conv_tc_c3_kernel(const ConvProblem p, const C3Geom g, const __grid_constant__ C
 
     if (warp < C::NISS) {
         // ------------------------------------------------------------------ MMA issuer of tiles n = warp (mod NISS), in order
-        constexpr uint32_t idesc = make_idesc(BN) | (1u << 10);                  // B operand: signed bytes
+        constexpr uint32_t idesc = make_idesc(AW) | (1u << 10);                  // B operand: signed bytes
+        constexpr uint32_t HALF_DESC = (uint32_t)(AW * ROWB) >> 4;               // weight rows of the second half
         const uint64_t desc0 = make_desc(wexp);
         const uint32_t desc_hi = (uint32_t)(desc0 >> 32), b_lo = (uint32_t)desc0;
         const uint32_t c_lo = (uint32_t)make_desc(cexp);
         const uint32_t tmem_u = __shfl_sync(0xffffffffu, tmem_base, 0);
         const uint32_t c_t = tmem_u + (uint32_t)C::C_COL;
-        for (int n = warp; n < my_tiles; n += C::NISS) {
-            const int acc = n % NACC;
+        bool ok = true;
+        for (int n = warp; n < my_tiles && ok; n += C::NISS) {
             if (!pw_wait(a_full(n % NAF), (uint32_t)(n / NAF) & 1u, abort_flag, p.err, ERR_C3_ISSUER_TIMEOUT)) break;
-            // the epilogue has read the accumulator's previous tile
-            if (n >= NACC && !pw_wait(acc_free(acc), (uint32_t)(n / NACC - 1) & 1u, abort_flag, p.err, ERR_C3_ACC_TIMEOUT)) break;
-            tc_fence_after();
-            if (elect_one()) {
-                const uint32_t d_t = tmem_u + (uint32_t)(acc * BN);
-                tc_mma_i8_ts(d_t, c_t, c_lo, desc_hi, idesc, 0u);               // accumulator = the per-channel constants
 #pragma unroll
-                for (int h = 0; h < CW; ++h) {
-                    const uint32_t a_t = tmem_u + (uint32_t)(C::A_COL0 + ((n * CW + h) % NUNIT) * U_COLS);
-#pragma unroll
-                    for (int t = 0; t < TAPS; ++t) {
-                        const int e = h * TAPS + t;
-                        tc_mma_i8_ts(d_t, a_t + 8u * t, b_lo + (uint32_t)((e >> 2) * (C::W_TILE_BYTES >> 4) + 2 * (e & 3)), desc_hi, idesc, 1u);
-                    }
+            for (int hf = 0; hf < NH; ++hf) {
+                // the epilogue has read the accumulator's previous tile
+                const int acc = NH == 2 ? hf : n % NACC;
+                const int prev = NH == 2 ? n - 1 : n / NACC - 1;                 // completion of acc_free to wait for
+                if (prev >= 0) {
+                    ok = pw_wait(acc_free(acc), (uint32_t)prev & 1u, abort_flag, p.err, ERR_C3_ACC_TIMEOUT);
+                    if (!ok) break;
                 }
-                tc_commit(tile_done(n % NB));
+                tc_fence_after();
+                if (elect_one()) {
+                    const uint32_t d_t = tmem_u + (uint32_t)(acc * AW);
+                    tc_mma_i8_ts(d_t, c_t, c_lo + hf * HALF_DESC, desc_hi, idesc, 0u);   // accumulator = the per-channel constants
+#pragma unroll
+                    for (int h = 0; h < CW; ++h) {
+                        const uint32_t a_t = tmem_u + (uint32_t)(C::A_COL0 + ((n * CW + h) % NUNIT) * U_COLS);
+#pragma unroll
+                        for (int t = 0; t < TAPS; ++t) {
+                            const int e = h * TAPS + t;
+                            tc_mma_i8_ts(d_t, a_t + 8u * t, b_lo + hf * HALF_DESC + (uint32_t)((e >> 2) * (C::W_TILE_BYTES >> 4) + 2 * (e & 3)),
+                                         desc_hi, idesc, 1u);
+                        }
+                    }
+                    tc_commit(tile_done((n * NH + hf) % NB));
+                }
+                __syncwarp();
             }
-            __syncwarp();
         }
     } else if (warp < C::FIRST_LOADER_WARP) {
         // (idle)
@@ -300,20 +316,23 @@ conv_tc_c3_kernel(const ConvProblem p, const C3Geom g, const __grid_constant__ C
         const int r = quad * 32 + lane;                           // row of the tile = output pixel (r / TW, r % TW)
         const uint32_t t_lane = tmem_base + ((uint32_t)(quad * 32) << 16);
         const int owords = p.C_out >> 5;
-        for (int n = grp; n < my_tiles; n += NGRP) {
-            const int acc = n % NACC;
-            if (!pw_wait<C::NISS == 1 ? 64 : 128>(tile_done(n % NB), (uint32_t)(n / NB) & 1u, abort_flag, p.err, ERR_C3_EPILOGUE_TIMEOUT)) break;
+        // NH == 1: the group takes alternate tiles; NH == 2: the group takes its half (64 channels) of every tile
+        for (int n = NH == 2 ? 0 : grp; n < my_tiles; n += NH == 2 ? 1 : NGRP) {
+            const int acc = NH == 2 ? grp : n % NACC;
+            const int d = NH == 2 ? 2 * n + grp : n;                              // the tile's (half's) "done" number
+            const int ch0 = NH == 2 ? 2 * grp : 0;                                // first output word of this accumulator
+            if (!pw_wait<C::NISS == 1 ? 64 : 128>(tile_done(d % NB), (uint32_t)(d / NB) & 1u, abort_flag, p.err, ERR_C3_EPILOGUE_TIMEOUT)) break;
             tc_fence_after();
-            uint32_t words[BN / 32];
+            uint32_t words[AW / 32];
             if constexpr (C::PACK16) {
-                constexpr int NR = BN == 32 ? 16 : 32;                       // registers per load
-                constexpr int NL = BN == 32 ? 1 : BN / 64;                   // loads
+                constexpr int NR = AW == 32 ? 16 : 32;                       // registers per load
+                constexpr int NL = AW == 32 ? 1 : AW / 64;                   // loads
                 uint32_t rr[NL][NR];
-                if constexpr (BN == 32) {
-                    tc_ld32_pack16(t_lane + (uint32_t)(acc * BN), rr[0]);
+                if constexpr (AW == 32) {
+                    tc_ld32_pack16(t_lane + (uint32_t)(acc * AW), rr[0]);
                 } else {
 #pragma unroll
-                    for (int h = 0; h < NL; ++h) tc_ld64_pack16(t_lane + (uint32_t)(acc * BN + h * 64), rr[h]);
+                    for (int h = 0; h < NL; ++h) tc_ld64_pack16(t_lane + (uint32_t)(acc * AW + h * 64), rr[h]);
                 }
                 tc_wait_ld();
 #pragma unroll
@@ -321,7 +340,7 @@ conv_tc_c3_kernel(const ConvProblem p, const C3Geom g, const __grid_constant__ C
                 tc_fence_before();
                 __syncwarp();
                 if (lane == 0) mbar_arrive(acc_free(acc));
-                if constexpr (BN == 32) {
+                if constexpr (AW == 32) {
                     words[0] = sign_word(rr[0]);
                 } else {
 #pragma unroll
@@ -332,40 +351,35 @@ conv_tc_c3_kernel(const ConvProblem p, const C3Geom g, const __grid_constant__ C
                 }
             } else {
 #pragma unroll
-                for (int ch = 0; ch < BN / 32; ++ch) {
-                    words[ch] = 0;
-                    if (ch * 32 < cn) {                                   // warp-uniform
-                        uint32_t v[32];
-                        tc_ld32(t_lane + (uint32_t)(acc * BN + ch * 32), v);
-                        if ((ch + 1) * 32 >= cn) {                        // the accumulator's last columns are in registers
-                            tc_fence_before();
-                            __syncwarp();
-                            if (lane == 0) mbar_arrive(acc_free(acc));
-                        }
-                        // bit i = (v[i] >= 0): sign bits shifted in, last column first; two chains of 16
-                        uint32_t hi = 0, lo = 0;
-#pragma unroll
-                        for (int i = 15; i >= 0; --i) {
-                            hi = __funnelshift_l(v[16 + i], hi, 1);
-                            lo = __funnelshift_l(v[i], lo, 1);
-                        }
-                        words[ch] = ~__byte_perm(lo, hi, 0x5410);
+                for (int ch = 0; ch < AW / 32; ++ch) {
+                    uint32_t v[32];
+                    tc_ld32(t_lane + (uint32_t)(acc * AW + ch * 32), v);
+                    if (ch == AW / 32 - 1) {                              // the accumulator's last columns are in registers
+                        tc_fence_before();
+                        __syncwarp();
+                        if (lane == 0) mbar_arrive(acc_free(acc));
                     }
+                    // bit i = (v[i] >= 0): sign bits shifted in, last column first; two chains of 16
+                    uint32_t hi = 0, lo = 0;
+#pragma unroll
+                    for (int i = 15; i >= 0; --i) {
+                        hi = __funnelshift_l(v[16 + i], hi, 1);
+                        lo = __funnelshift_l(v[i], lo, 1);
+                    }
+                    words[ch] = ~__byte_perm(lo, hi, 0x5410);
                 }
             }
             int b, oh0, ow0;
             tile_origin(tile_of(n), b, oh0, ow0);
             const int oh = oh0 + (r >> 4), ow = ow0 + (r & 15);
             if (oh < p.OH && ow < p.OW) {
-                uint32_t *dst = static_cast<uint32_t *>(p.out) + (((long)b * p.OH + oh) * p.OW + ow) * owords;
-                if (BN == 128 && owords == 4) {
-                    *reinterpret_cast<uint4 *>(dst) = make_uint4(words[0], words[1 % (BN / 32)], words[2 % (BN / 32)], words[3 % (BN / 32)]);
-                } else if (BN >= 64 && owords == 2) {
-                    *reinterpret_cast<uint2 *>(dst) = make_uint2(words[0], words[1 % (BN / 32)]);
+                uint32_t *dst = static_cast<uint32_t *>(p.out) + (((long)b * p.OH + oh) * p.OW + ow) * owords + ch0;
+                if (AW == 64 && (owords & 1) == 0) {                  // (an even word count keeps the pair 8-byte aligned)
+                    *reinterpret_cast<uint2 *>(dst) = make_uint2(words[0], words[1 % (AW / 32)]);
                 } else {
 #pragma unroll
-                    for (int ch = 0; ch < BN / 32; ++ch)
-                        if (ch < owords) dst[ch] = words[ch];
+                    for (int ch = 0; ch < AW / 32; ++ch)
+                        if (ch0 + ch < owords) dst[ch] = words[ch];
                 }
             }
         }
@@ -400,8 +414,8 @@ conv_tc_c3_kernel(const ConvProblem p, const C3Geom g, const __grid_constant__ C
             // the MMAs of the tile that used this ring position last have read it (nothing to wait for the first time round)
             const int u = n * CW + h;
             if (u >= NUNIT) {
-                const int m = (u - NUNIT) / CW;
-                if (!pw_wait<64>(tile_done(m % NB), (uint32_t)(m / NB) & 1u, abort_flag, p.err, ERR_C3_UNIT_TIMEOUT)) break;
+                const int dm = (u - NUNIT) / CW * NH + NH - 1;                    // that tile's last "done" number
+                if (!pw_wait<64>(tile_done(dm % NB), (uint32_t)(dm / NB) & 1u, abort_flag, p.err, ERR_C3_UNIT_TIMEOUT)) break;
             }
             tc_fence_after();
             const uint32_t taddr = t_lane + (uint32_t)((u % NUNIT) * U_COLS);
