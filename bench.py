@@ -530,6 +530,7 @@ def run_gpu(args):
                  "tc_pw": "conv_tc_pw_kernel (tcgen05 kind::i8, pointwise layers, bulk-copied rows)",
                  "tc_pre": "conv_tc_pre_kernel (tcgen05 kind::i8, prepared weights streamed by TMA)",
                  "tc_c3": "conv_tc_c3_kernel (tcgen05 kind::i8, 3x3 layers on 32/64 channels, halo tiles by TMA)",
+                 "tc_pn": "conv_tc_pn_kernel (tcgen05 kind::i8, pointwise layers with K = 256 / 512, resident weight slices)",
                  "lop3": "conv_k32_kernel (CUDA-core xor + popc)"}
     lay_ms = [float(per_ms[0]) if engines[i] == "stem" else float(per_ms[i + 1]) for i in range(nl)]
     per_layer = []
@@ -561,7 +562,8 @@ def run_gpu(args):
     top_tops = lt.ops(B) / (per_ms[top + 1] / 1e3) / 1e12
     src_of = {"tc_ws": ["conv_tc_ws.cu", "tc_common.cuh"], "tc_i8": ["conv_tc_i8.cu", "tc_common.cuh"],
               "tc_pw": ["conv_tc_pw.cu", "tc_slot.cuh", "tc_common.cuh"], "tc_pre": ["conv_tc_pre.cu", "tc_common.cuh"],
-              "tc_c3": ["conv_tc_c3.cu", "tc_slot.cuh", "tc_common.cuh"]}
+              "tc_c3": ["conv_tc_c3.cu", "tc_slot.cuh", "tc_common.cuh"],
+              "tc_pn": ["conv_tc_pn.cu", "tc_slot.cuh", "tc_common.cuh"]}
     roofline = {
         "kernel": groups[0]["kernel"], "launch": f"{lt.name}: M={lt.M(B)} N={lt.C_out} K={lt.K}",
         "bound": "tensor", "achieved": top_tops, "peak": tensor_peak, "unit": "TOP/s", "frac": top_tops / tensor_peak,
@@ -890,7 +892,7 @@ def run_block(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--mode", default="bench", choices=["bench", "sweep", "paper1x1", "block"])
-    ap.add_argument("--engines", default="auto,lop3,mma_b1,tc_i8,mma_s8,tc_ws,tc_pw,tc_c3,tc_pre")
+    ap.add_argument("--engines", default="auto,lop3,mma_b1,tc_i8,mma_s8,tc_ws,tc_pw,tc_c3,tc_pn,tc_pre")
     ap.add_argument("--sweep-set", default="all", choices=["gemm", "conv", "all", "paper"])
     ap.add_argument("--only", default="", help="sweep mode: run only shapes whose label contains this text")
     ap.add_argument("--outs", default="int32,fused", help="sweep mode: output kinds to run")

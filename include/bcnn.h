@@ -61,9 +61,12 @@ typedef enum bcnn_engine {
     BCNN_ENGINE_TC_WS = 5,  /* tcgen05 kind::i8 with the expanded weight tile resident in shared memory (C_out <= 128) */
     BCNN_ENGINE_TC_PW = 6,  /* tcgen05 kind::i8 for pointwise layers (1x1, stride 1, no padding; GEMMs) with K <= 128 and
                                C_out <= 128, packed output: rows bulk-copied in chunks, one hand-over per chunk */
-    BCNN_ENGINE_TC_C3 = 7   /* tcgen05 kind::i8 for 3x3 layers (stride 1 or 2, padding 0 or 1) on 32 or 64 input channels
+    BCNN_ENGINE_TC_C3 = 7,  /* tcgen05 kind::i8 for 3x3 layers (stride 1 or 2, padding 0 or 1) on 32 or 64 input channels
                                with C_out <= 128 and W * C_in a multiple of 128, packed output: the input halo of an
                                8 x 16 tile of output pixels arrives by one tiled TMA copy, padding is the copy's zero fill */
+    BCNN_ENGINE_TC_PN = 8   /* tcgen05 kind::i8 for pointwise layers (1x1, stride 1, no padding; GEMMs) with K = 256 or 512 and
+                               128, 256 or 512 output channels, packed output: a row tile is expanded once and multiplied
+                               against all the weight slices a CTA keeps in shared memory */
 } bcnn_engine;
 
 /*

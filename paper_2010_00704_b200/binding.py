@@ -15,9 +15,9 @@ import torch
 _PKG = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_PKG, "libbcnn.so")
 
-ENGINE_AUTO, ENGINE_LOP3, ENGINE_MMA_B1, ENGINE_TC_I8, ENGINE_MMA_S8, ENGINE_TC_WS, ENGINE_TC_PW, ENGINE_TC_C3 = 0, 1, 2, 3, 4, 5, 6, 7
+ENGINE_AUTO, ENGINE_LOP3, ENGINE_MMA_B1, ENGINE_TC_I8, ENGINE_MMA_S8, ENGINE_TC_WS, ENGINE_TC_PW, ENGINE_TC_C3, ENGINE_TC_PN = 0, 1, 2, 3, 4, 5, 6, 7, 8
 ENGINES = {"auto": ENGINE_AUTO, "lop3": ENGINE_LOP3, "mma_b1": ENGINE_MMA_B1, "tc_i8": ENGINE_TC_I8,
-           "mma_s8": ENGINE_MMA_S8, "tc_ws": ENGINE_TC_WS, "tc_pw": ENGINE_TC_PW, "tc_c3": ENGINE_TC_C3}
+           "mma_s8": ENGINE_MMA_S8, "tc_ws": ENGINE_TC_WS, "tc_pw": ENGINE_TC_PW, "tc_c3": ENGINE_TC_C3, "tc_pn": ENGINE_TC_PN}
 
 EXPORTS = (
     "bcnn_pack", "bcnn_stem_fused", "bcnn_gemm_b1", "bcnn_gemm_b1_fused", "bcnn_conv2d_b1", "bcnn_conv2d_b1_fused", "bcnn_conv2d_b1_module",

@@ -76,6 +76,8 @@ int make_conv_problem(ConvProblem &p, const void *x, const void *w, const int32_
 // Measured on B200 (bench.py --mode sweep):
 //   * pointwise layers (1x1, stride 1, no padding; GEMMs) with K <= 128 and C_out <= 128, packed output: pointwise
 //     tcgen05 engine (memory-bound shapes: rows bulk-copied in chunks, one hand-over per chunk);
+//   * pointwise layers with K = 256 or 512 and 128, 256 or 512 output channels, packed output: wide pointwise tcgen05
+//     engine (a row tile expanded once for all resident weight slices; 1.2 - 2x the weight-stationary engine);
 //   * 3x3 layers (stride 1 or 2) on 32 or 64 input channels with C_out <= 64, packed output, whose 8 x 16 output tiles
 //     are at least three quarters full: halo-tile tcgen05 engine (input tiles by tiled TMA copies);
 //   * C_out >= 256, or weights too large to keep expanded in shared memory: streaming tcgen05 engine;
@@ -87,6 +89,7 @@ int make_conv_problem(ConvProblem &p, const void *x, const void *w, const int32_
 int auto_engine(const ConvProblem &p)
 {
     if (conv_tc_pw_supports(p)) return BCNN_ENGINE_TC_PW;
+    if (conv_tc_pn_supports(p)) return BCNN_ENGINE_TC_PN;
     if (p.C_out <= 64 && conv_tc_c3_supports(p)) {
         const long covered = (long)((p.OH + 7) / 8 * 8) * ((p.OW + 15) / 16 * 16);
         if (4L * p.OH * p.OW >= 3L * covered) return BCNN_ENGINE_TC_C3;
@@ -120,6 +123,8 @@ int dispatch(int engine, const ConvProblem &p, cudaStream_t stream)
         return launch_conv_tc_pw(p, stream);
     case BCNN_ENGINE_TC_C3:
         return launch_conv_tc_c3(p, stream);
+    case BCNN_ENGINE_TC_PN:
+        return launch_conv_tc_pn(p, stream);
     default:
         return BCNN_ERR_UNSUPPORTED;
     }
@@ -459,6 +464,12 @@ const char *bcnn_status_string(int status)
     case 144: return "device wait timed out: 3x3 halo-tile tcgen05 engine, epilogue waiting for a tile's accumulator";
     case 145: return "device wait timed out: 3x3 halo-tile tcgen05 engine, producer waiting for an activation stage's previous MMAs";
     case 146: return "device wait timed out: 3x3 halo-tile tcgen05 engine, issuer waiting for an accumulator";
+    case 151: return "device wait timed out: wide pointwise tcgen05 engine, loader waiting for a free ring stage";
+    case 152: return "device wait timed out: wide pointwise tcgen05 engine, producer waiting for a tile's rows";
+    case 153: return "device wait timed out: wide pointwise tcgen05 engine, issuer waiting for a tile's expanded rows";
+    case 154: return "device wait timed out: wide pointwise tcgen05 engine, epilogue waiting for an accumulator";
+    case 155: return "device wait timed out: wide pointwise tcgen05 engine, producer waiting for an activation unit's previous MMAs";
+    case 156: return "device wait timed out: wide pointwise tcgen05 engine, issuer waiting for an accumulator";
     case BCNN_SELFTEST_TIMEOUT_CODE: return "device wait timed out: self-test (expected)";
     default: return status > 0 ? "device-side error code" : "unknown status";
     }

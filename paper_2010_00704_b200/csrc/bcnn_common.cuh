@@ -96,6 +96,8 @@ int launch_conv_tc_pw(const ConvProblem &p, cudaStream_t stream);
 bool conv_tc_pw_supports(const ConvProblem &p);
 int launch_conv_tc_c3(const ConvProblem &p, cudaStream_t stream);
 bool conv_tc_c3_supports(const ConvProblem &p);
+int launch_conv_tc_pn(const ConvProblem &p, cudaStream_t stream);
+bool conv_tc_pn_supports(const ConvProblem &p);
 int launch_conv_tc_i8(const ConvProblem &p, cudaStream_t stream);
 // weights expanded once per layer by launch_prepare_weights (conv_tc_pre.cu): [n_pad][k_pad] signed bytes, then
 // K - 2 popc(W_n) per row

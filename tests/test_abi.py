@@ -31,7 +31,7 @@ def test_status_strings_and_version():
     assert "workspace" in binding.status_string(binding.ERR_WORKSPACE)
     assert "wait" in binding.status_string(binding.ERR_TIMEOUT)
     # the device error codes name the engine and the role whose wait gave up
-    for code in (101, 102, 103, 111, 112, 113, 121, 122, 123, 124, 125, 126, 131, 132, 133, 134, 141, 142, 143, 144, 145, 146,
+    for code in (101, 102, 103, 111, 112, 113, 121, 122, 123, 124, 125, 126, 131, 132, 133, 134, 141, 142, 143, 144, 145, 146, 151, 152, 153, 154, 155, 156,
                  binding.SELFTEST_TIMEOUT_CODE):
         assert "timed out" in binding.status_string(code)
     assert binding.status_string(77) == "device-side error code"

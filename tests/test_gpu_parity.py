@@ -17,7 +17,7 @@ def bk():
     return binding
 
 
-ENGINES = ["auto", "lop3", "mma_b1", "tc_i8", "mma_s8", "tc_ws", "tc_pw", "tc_c3"]
+ENGINES = ["auto", "lop3", "mma_b1", "tc_i8", "mma_s8", "tc_ws", "tc_pw", "tc_c3", "tc_pn"]
 
 
 def dev(a):
@@ -104,6 +104,12 @@ CONV_SHAPES = [
     (1, 50, 40, 32, 96, 3, 3, 1, 0),       # ... 96 of 128 accumulator columns, no padding
     (1, 41, 48, 64, 128, 3, 3, 2, 1),      # ... two-word pixels, 128 channels: one accumulator
     (1, 30, 34, 64, 64, 3, 3, 1, 1),       # ... image rows of 68 words: W * C_in / 32 is a multiple of 4, W is not
+    (2, 29, 31, 256, 256, 1, 1, 1, 0),     # wide pointwise engine: K = 256, two parts per tile, ragged last tile
+    (1, 37, 41, 256, 128, 1, 1, 1, 0),     # ... one part per tile (one of the two issuers idles)
+    (1, 23, 19, 256, 512, 1, 1, 1, 0),     # ... four resident slices
+    (1, 33, 35, 512, 512, 1, 1, 1, 0),     # ... K = 512: two units per tile, four CTA groups of one slice
+    (1, 21, 22, 512, 256, 1, 1, 1, 0),     # ... two CTA groups
+    (1, 11, 13, 512, 128, 1, 1, 1, 0),     # ... one group, two parts of 64 channels
 ]
 
 
@@ -167,7 +173,7 @@ def test_conv_constant_inputs(bk, engine):
     K = 9 * Ci
     xm = -np.ones((B, H, W, Ci), np.int8)
     wp = np.ones((Co, 3, 3, Ci), np.int8)
-    if engine in ("tc_pw", "tc_c3"):
+    if engine in ("tc_pw", "tc_c3", "tc_pn"):
         pytest.skip("the pointwise and halo-tile engines have packed output only")
     assert np.all(run_conv(bk, xm, wp, None, 1, 1, engine) == -K)
     assert np.all(run_conv(bk, xm, -wp, None, 2, 1, engine) == K)
@@ -214,7 +220,40 @@ def test_tc_c3_many_tiles_sampled(bk, oracle, shape):
     assert torch.equal(ref, buf)                       # (the other engine is itself checked against the oracle above)
 
 
-GEMM_SHAPES = [(1024, 1024, 512), (1024, 1024, 2304), (300, 200, 96), (129, 33, 1056), (64, 512, 4608), (1, 32, 32)]
+@pytest.mark.parametrize("shape", [
+    (333 * 128 + 77, 512, 512),       # nine and ten row tiles per CTA (four groups of 37): every ring and barrier ring wraps
+    (148 * 9 * 128 + 5, 256, 256),    # K = 256: ten tiles per CTA
+    (50000, 128, 512),
+    (70001, 512, 256),
+])
+def test_tc_pn_many_tiles_sampled(bk, oracle, shape):
+    """The wide pointwise engine over many tiles per CTA, against the oracle on sampled rows (the first and last ones,
+    the rows around tile borders, random ones) and against the weight-stationary engine everywhere."""
+    M, N, K = shape
+    rng = np.random.default_rng(31 + sum(shape))
+    Ab = synth.random_bits(rng, (M, K // 8))
+    Wb = synth.random_bits(rng, (N, K // 8))
+    thr = plant_extreme_thresholds(synth.thresholds(rng, K, N), K)
+    dA, dW, dthr = dev(Ab), dev(Wb), dev(thr)
+    raw, ob = guard_alloc(M * N // 8)
+    bk.bcnn_gemm_b1_fused(dA, dW, dthr, ob, M, N, K, engine=bk.ENGINES["tc_pn"])
+    torch.cuda.synchronize()
+    assert bk.bcnn_device_error() == 0
+    check_guards(raw, M * N // 8)
+    got = synth.unpack_bits(ob.cpu().numpy().reshape(M, N // 8))
+    rows = {0, 1, 127, 128, 129, M - 130, M - 129, M - 128, M - 2, M - 1}
+    rows.update(int(v) for v in rng.integers(0, M, 1500))
+    rows = np.array(sorted(rows), dtype=np.int64)
+    want = oracle.threshold(oracle.gemm(synth.unpack_bits(Ab[rows]), synth.unpack_bits(Wb)), thr)
+    assert np.array_equal(got[rows], want)
+    ref = torch.zeros(M * N // 8, dtype=torch.uint8, device="cuda")
+    bk.bcnn_gemm_b1_fused(dA, dW, dthr, ref, M, N, K, engine=bk.ENGINES["tc_ws"])
+    torch.cuda.synchronize()
+    assert torch.equal(ref, ob)                        # (the other engine is itself checked against the oracle above)
+
+
+GEMM_SHAPES = [(1024, 1024, 512), (1024, 1024, 2304), (300, 200, 96), (129, 33, 1056), (64, 512, 4608), (1, 32, 32),
+               (3000, 256, 256), (1, 128, 512), (2049, 512, 256)]
 
 
 @pytest.mark.parametrize("engine", ENGINES)
