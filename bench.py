@@ -764,6 +764,11 @@ def run_paper1x1(args):
                 nb = torch.from_numpy(synth.real_input(rng, (l.C_out,))).cuda()
                 sl = torch.from_numpy(rng.uniform(0.0, 0.5, l.C_out).astype(np.float32)).cuda()
                 extra = (sc, sh, ident, sl, nb, yreal)
+            elif binding.bcnn_prepared_preferred(B, l.H, l.W, l.C_in, l.C_out, 1, 1, 1, 0):
+                # as FusedChain does: a layer's weights are expanded once, at set-up, where the library prefers that
+                prep = torch.empty(binding.bcnn_prepared_weights_bytes(l.C_out, l.K), dtype=torch.uint8, device="cuda")
+                binding.bcnn_prepare_weights(Wb, prep, l.C_out, l.K)
+                extra = prep
             jobs.append((l, x, Wb, thr, out, extra))
 
     def launch(j):
@@ -774,6 +779,8 @@ def run_paper1x1(args):
                 binding.bcnn_conv2d_b1_branches(x, Wb, sc, sh, None, idn, sl, nb, yr, out, B, l.H, l.W, l.C_in, l.C_out, P)
             else:
                 binding.bcnn_conv2d_b1_module(x, Wb, sc, sh, idn, sl, nb, yr, out, B, l.H, l.W, l.C_in, l.C_out, 1, 1, 1, 0)
+        elif extra is not None:
+            binding.bcnn_conv2d_b1_prepared(x, extra, thr, out, B, l.H, l.W, l.C_in, l.C_out, 1, 1, 1, 0)
         else:
             binding.bcnn_conv2d_b1_fused(x, Wb, thr, out, B, l.H, l.W, l.C_in, l.C_out, 1, 1, 1, 0)
 
@@ -815,7 +822,8 @@ def run_paper1x1(args):
         ms = float(np.mean([a.elapsed_time(b) for a, b in per[l.name]]))
         shapes.append({"layer": l.name, "count": count, "M": l.M(B), "N": l.C_out, "K": l.K,
                        "engine": ("branches (CUDA cores)" if branch_call else "tc_ws") if module
-                       else binding.bcnn_auto_engine(B, l.H, l.W, l.C_in, l.C_out, 1, 1, 1, 0),
+                       else ("tc_pre" if binding.bcnn_prepared_preferred(B, l.H, l.W, l.C_in, l.C_out, 1, 1, 1, 0)
+                             else binding.bcnn_auto_engine(B, l.H, l.W, l.C_in, l.C_out, 1, 1, 1, 0)),
                        "ms_per_launch": ms, "tops": PB * l.ops(B) / (ms / 1e3) / 1e12})
         # algorithmic bytes: packed input + packed output (+ fp16 identity read and fp16 map written by the module)
         nbytes = PB * l.in_bytes(B) + l.out_bits_bytes(B) + (4 * l.M(B) * l.C_out if module else 0)

@@ -118,12 +118,19 @@ conv_tc_pn_kernel(const ConvProblem p, const PnPlan plan)
         abort_flag_smem = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
+    __syncthreads();
+    // The loader warps start now: the first row tiles arrive while the other warps expand the weights (these kernels
+    // run for 10 - 40 us; the weights' expansion and the first copy's latency are 1.5 - 2 us each).  The other warps meet
+    // at a named barrier of their own; everybody meets again at the end.
+    const bool is_loader = warp >= FIRST_LOADER_WARP && warp < FIRST_PRODUCER_WARP;
+    auto sync_workers = [&]() { asm volatile("bar.sync 1, %0;" ::"r"(THREADS - 64) : "memory"); };
+    if (!is_loader) {
     if (warp == 0) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_smem)), "r"(512u) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
     // ---- one-off: the resident slices' expanded weights and constants; MMA row `row` of slice s carries channel ch
-    for (int i = tid; i < RS * (KT + 1) * BN; i += THREADS) {
+    for (int i = tid < 64 ? tid : tid - 64; i < RS * (KT + 1) * BN; i += THREADS - 64) {   // (threads 64 .. 127 are the loaders)
         const int row = i % BN, kt = (i / BN) % (KT + 1), s = i / (BN * (KT + 1));
         const int ch = (cg * RS + s) * BN + (PACK16 ? (row & ~31) + channel_of_column(row & 31) : row);
         const bool have = ch < p.C_out;
@@ -160,18 +167,19 @@ conv_tc_pn_kernel(const ConvProblem p, const PnPlan plan)
     }
     fence_async_proxy();
     tc_fence_before();
-    __syncthreads();
+    sync_workers();
     tc_fence_after();
-    const uint32_t tmem_base = tmem_base_smem;
     // the constant activation tile: every byte 32
     if (warp >= FIRST_PRODUCER_WARP && warp < FIRST_PRODUCER_WARP + 4) {
         const uint32_t c8[8] = {0x20202020u, 0x20202020u, 0x20202020u, 0x20202020u, 0x20202020u, 0x20202020u, 0x20202020u, 0x20202020u};
-        tc_st8_nowait(tmem_base + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)C_COL, c8);
+        tc_st8_nowait(tmem_base_smem + ((uint32_t)((warp & 3) * 32) << 16) + (uint32_t)C_COL, c8);
         tc_wait_st();
     }
     tc_fence_before();
-    __syncthreads();
+    sync_workers();
     tc_fence_after();
+    }
+    const uint32_t tmem_base = is_loader ? 0u : tmem_base_smem;
 
     if (warp < NISS) {
         // ------------------------------------------------------------------ MMA issuer of the parts d = warp (mod 2), in order.
